@@ -1,0 +1,439 @@
+#!/usr/bin/env python
+"""Benchmark of the B200 FFT / SAR library.
+
+Metric: batched FFT effective GB/s = (bytes in + bytes out) / time, cold cache
+(every batch is far larger than the 126 MB L2), on the workload
+"N=4096, batch=32768 complex64, contiguous, forward". One step = one
+fft_execute over the whole batch. Also reported in the same JSON line: the other
+workloads (N=8192/16384 in fp32 and fp16 storage, 4096^2 column and 2-D
+transforms, the 4096^2 range-Doppler SAR image in ms), the end-to-end number
+with host buffers, the roofline fraction of the dominant kernel, and the CPU
+oracle timed on this machine.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--only main]
+
+For N > 1 launch under torch.distributed.run; every rank processes its own
+batch of the same size (weak scaling, no data-path collective).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2609_32237_b200 import inputs, metrics  # noqa: E402
+
+MAIN = dict(n=4096, batch=32768, seed=1, dtype=0)
+WORKLOAD = "N=4096 batch=32768 complex64 forward, contiguous rows (1 GiB in + 1 GiB out)"
+
+
+# ----------------------------------------------------------------------------- helpers
+def measured_peak_gbs():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        try:
+            return float(json.load(open(p))["hbm_gbs"]), "measured"
+        except Exception:
+            pass
+    return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}",
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=2)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], None, set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            parts = [p.strip() for p in ln.split(",")]
+            if len(parts) < 6:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                mx = float(parts[1])
+            except ValueError:
+                continue
+            for nm, val in zip(names, parts[2:6]):
+                if val.lower().startswith("active"):
+                    reasons.add(nm)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": mx,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def dist_env():
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    return rank, world, local
+
+
+# ----------------------------------------------------------------------------- reference arm (CPU oracle)
+def run_reference(args):
+    rank, world, _ = dist_env()
+    if rank != 0:
+        return 0
+    import oracle
+    n, sample = MAIN["n"], 4096
+    x = inputs.gaussian_complex64((sample, n), MAIN["seed"]).astype(np.complex128)
+    for _ in range(args.warmup):
+        oracle.fft_rows(x[:256])
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle.fft_rows(x)
+    dt = (time.perf_counter() - t0) / args.steps
+    gbs = metrics.fft_bytes(n, sample, 0) / dt / 1e9
+    cores = oracle.num_threads()
+    line = {
+        "impl": "reference", "metric": "batched FFT effective GB/s", "value": gbs, "unit": "GB/s",
+        "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "data": "synthetic", "config": {"workload": WORKLOAD, "sample": f"{sample} of 32768 transforms per step"},
+        "cpu_baseline": {"value": gbs, "unit": "GB/s", "cores": cores, "kind": "oracle",
+                         "sample": f"{sample} transforms of N={n} per step (float64 recursive radix-2)"},
+        "e2e": {"value": gbs, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+    return 0
+
+
+# ----------------------------------------------------------------------------- GPU arm
+def time_calls(torch, fn, steps, warmup, stream):
+    """Device time of `steps` calls of fn() on `stream`, warm-up first; returns
+    (total ms, per-call ms list)."""
+    for _ in range(warmup):
+        fn()
+    torch.cuda.synchronize()
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+    for a, b in evs:
+        a.record(stream)
+        fn()
+        b.record(stream)
+    torch.cuda.synchronize()
+    per = [a.elapsed_time(b) for a, b in evs]
+    return sum(per), per
+
+
+def flush_l2(torch, scratch):
+    scratch.zero_()
+
+
+def bench_fft(torch, B, n, batch, dtype, seed, steps, warmup, layout="rows", direction=-1, cold_flush=None):
+    stream = torch.cuda.current_stream()
+    if layout == "rows":
+        x = inputs.gaussian_complex64((batch, n), seed)
+        plan = B.fft_plan_create(n, batch, 1, n, direction, dtype)
+    else:
+        x = inputs.uniform_complex64((n, batch), seed)
+        plan = B.fft_plan_create(n, batch, batch, 1, direction, dtype)
+    if dtype == 0:
+        d_in = torch.from_numpy(x).cuda()
+    else:
+        d_in = torch.from_numpy(inputs.to_half_storage(x)).cuda()
+    del x
+    d_out = torch.empty_like(d_in)
+    need = B.fft_plan_workspace_bytes(plan)
+    ws = None
+    if need:
+        ws = torch.empty(need, dtype=torch.uint8, device="cuda")
+        B.fft_plan_set_workspace(plan, ws.data_ptr(), need)
+
+    def call():
+        if cold_flush is not None:
+            flush_l2(torch, cold_flush)
+        B.fft_execute(plan, d_in.data_ptr(), d_out.data_ptr(), stream.cuda_stream)
+
+    if cold_flush is None:
+        total, per = time_calls(torch, call, steps, warmup, stream)
+    else:
+        # flush outside the event pair
+        for _ in range(warmup):
+            call()
+        torch.cuda.synchronize()
+        per = []
+        for _ in range(steps):
+            flush_l2(torch, cold_flush)
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            B.fft_execute(plan, d_in.data_ptr(), d_out.data_ptr(), stream.cuda_stream)
+            b.record(stream)
+            torch.cuda.synchronize()
+            per.append(a.elapsed_time(b))
+        total = sum(per)
+    B.fft_plan_destroy(plan)
+    return total, per, (d_in, d_out)
+
+
+def summarize(per_ms, nbytes, peak):
+    med = float(np.median(per_ms))
+    q1, q3 = np.percentile(per_ms, [25, 75])
+    gbs = nbytes / (med * 1e-3) / 1e9
+    return {"ms_median": med, "ms_min": float(min(per_ms)), "ms_iqr": float(q3 - q1),
+            "gbs": gbs, "frac_of_peak": gbs / peak}
+
+
+def run_gpu(args):
+    import torch
+    rank, world, local = dist_env()
+    if world > 1:
+        import torch.distributed as dist
+        torch.cuda.set_device(local)
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    else:
+        torch.cuda.set_device(0)
+    from paper_2609_32237_b200 import binding as B   # fails loudly if the CUDA library is missing
+    peak, peak_kind = measured_peak_gbs()
+    stream = torch.cuda.current_stream()
+    n, batch, dtype = MAIN["n"], MAIN["batch"], MAIN["dtype"]
+    nbytes = metrics.fft_bytes(n, batch, dtype)
+
+    # ---- main workload: inputs resident in HBM ---------------------------------
+    x = inputs.gaussian_complex64((batch, n), MAIN["seed"] + rank)
+    h_in = torch.from_numpy(x).pin_memory()
+    h_out = torch.empty_like(h_in).pin_memory()
+    d_in = h_in.cuda()
+    d_out = torch.empty_like(d_in)
+    plan = B.fft_plan_create(n, batch, 1, n, -1, dtype)
+
+    def step():
+        B.fft_execute(plan, d_in.data_ptr(), d_out.data_ptr(), stream.cuda_stream)
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    launches0 = B.launch_count()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(args.steps):
+        step()
+    e1.record(stream)
+    torch.cuda.synchronize()
+    total_ms = e0.elapsed_time(e1)
+    launches = B.launch_count() - launches0
+    if world > 1:
+        t = torch.tensor([total_ms], device="cuda", dtype=torch.float64)
+        dist.barrier()
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    clocks = sampler.stop() if rank == 0 else None
+    ms_per_step = total_ms / args.steps
+    value = world * nbytes / (ms_per_step * 1e-3) / 1e9
+    kernel_gbs = nbytes / (ms_per_step * 1e-3) / 1e9     # one launch per step: launch duration = step time
+
+    # ---- end to end: host buffers, copies inside the timed region ------------------
+    def step_host():
+        B.fft_execute_host(plan, h_in.data_ptr(), h_out.data_ptr(), d_in.data_ptr(), d_out.data_ptr(),
+                           stream.cuda_stream)
+
+    e2e_steps = max(2, min(args.steps, 5))
+    step_host()
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    e0.record(stream)
+    for _ in range(e2e_steps):
+        step_host()
+    e1.record(stream)
+    torch.cuda.synchronize()
+    e2e_ms = e0.elapsed_time(e1)
+    if world > 1:
+        t = torch.tensor([e2e_ms], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_ms = float(t.item())
+    e2e_value = world * nbytes / (e2e_ms / e2e_steps * 1e-3) / 1e9
+    checksum = float(h_out.view(torch.float32)[:8].abs().sum())
+    B.fft_plan_destroy(plan)
+    del d_in, d_out, h_in, h_out, x
+    torch.cuda.empty_cache()
+
+    line = {
+        "metric": "batched FFT effective GB/s", "value": value, "unit": "GB/s", "n_gpus": world,
+        "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+        "data": "synthetic",
+        "config": {"workload": WORKLOAD, "cold_cache": "inputs larger than L2 (2 GiB touched per step vs 126 MB)",
+                   "parallelism": f"replicas x{world}" if world > 1 else "1 gpu"},
+        "pct_of_hbm_peak": 100.0 * kernel_gbs / peak, "gflops": metrics.fft_gflops(n, batch, ms_per_step * 1e-3) * world,
+        "e2e": {"value": e2e_value, "unit": "GB/s", "h2d_bytes_per_step": nbytes // 2, "d2h_bytes_per_step": nbytes // 2,
+                "steps": e2e_steps, "checksum": checksum},
+        "gpu_launches": int(launches),
+        "clocks": clocks,
+        "roofline": {"bound": "hbm", "achieved": kernel_gbs, "peak": peak, "unit": "GB/s",
+                     "frac": kernel_gbs / peak, "traffic": metrics.NCU_TRAFFIC_BYTES.get("fft_rows_4096_c64"),
+                     "peak_kind": f"of {peak_kind}", "algorithmic_bytes": nbytes,
+                     "kernel": "fft_kernel<N=4096, rows, c64>"},
+    }
+
+    if rank == 0 and not args.only_main:
+        line["others"] = run_others(torch, B, args, peak)
+    if rank == 0:
+        line["cpu_baseline"] = cpu_baseline(n)
+        print(json.dumps(line))
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+    return 0
+
+
+def run_others(torch, B, args, peak):
+    """Every other workload, each timed cold (a 512 MiB scratch write before each
+    sample, outside the event pair) with its own warm-up."""
+    steps, warmup = max(5, min(args.steps, 15)), 3
+    scratch = torch.empty(512 << 20, dtype=torch.uint8, device="cuda")
+    out = {}
+
+    def fft_case(name, n, batch, dtype, seed, layout="rows", direction=-1):
+        _, per, _ = bench_fft(torch, B, n, batch, dtype, seed, steps, warmup, layout, direction, cold_flush=scratch)
+        s = summarize(per, metrics.fft_bytes(n, batch, dtype), peak)
+        s["gflops"] = metrics.fft_gflops(n, batch, s["ms_median"] * 1e-3)
+        out[name] = s
+        torch.cuda.empty_cache()
+
+    fft_case("fft_n4096_b32768_c64_inverse", 4096, 32768, 0, 1, direction=1)
+    fft_case("fft_n8192_b16384_c64", 8192, 16384, 0, 2)
+    fft_case("fft_n16384_b8192_c64", 16384, 8192, 0, 2)
+    fft_case("fft_n8192_b16384_c32h", 8192, 16384, 1, 2)
+    fft_case("fft_n16384_b8192_c32h", 16384, 8192, 1, 2)
+    fft_case("fft_n1024_b256_c64", 1024, 256, 0, 0)
+    fft_case("fft_cols_4096x4096_c64", 4096, 4096, 0, 3, layout="cols")
+    fft_case("fft_n65536_b2048_c64_four_step", 65536, 2048, 0, 5)
+    out["fft_n65536_b2048_c64_four_step"]["note"] = "two passes: algorithmic bytes counted once (16 B/point)"
+
+    # 2-D: rows then columns, in place
+    stream = torch.cuda.current_stream()
+    m = torch.from_numpy(inputs.uniform_complex64((4096, 4096), 3)).cuda()
+    pr = B.fft_plan_create(4096, 4096, 1, 4096, -1, 0)
+    pc = B.fft_plan_create(4096, 4096, 4096, 1, -1, 0)
+    per = []
+    for i in range(warmup + steps):
+        flush_l2(torch, scratch)
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        B.fft_execute(pr, m.data_ptr(), m.data_ptr(), stream.cuda_stream)
+        B.fft_execute(pc, m.data_ptr(), m.data_ptr(), stream.cuda_stream)
+        b.record(stream)
+        torch.cuda.synchronize()
+        if i >= warmup:
+            per.append(a.elapsed_time(b))
+    B.fft_plan_destroy(pr)
+    B.fft_plan_destroy(pc)
+    out["fft2d_4096x4096_c64"] = summarize(per, 2 * metrics.fft_bytes(4096, 4096, 0), peak)
+
+    # SAR
+    sc = inputs.x_band_scene()
+    raw = inputs.simulate_raw(sc, seed=4)
+    rd = torch.from_numpy(raw).cuda()
+    img = torch.empty_like(rd)
+    for dtype, name in ((0, "sar_4096x4096_fp32_intermediates"), (1, "sar_4096x4096_fp16_intermediates")):
+        p = B.sar_rda_params_create(B.sar_desc_from_scene(sc, dtype))
+        need = B.sar_rda_workspace_bytes(p)
+        ws = torch.empty(need, dtype=torch.uint8, device="cuda")
+        B.sar_rda_set_workspace(p, ws.data_ptr(), need)
+        per, per_step = [], [[], [], []]
+        for i in range(warmup + steps):
+            flush_l2(torch, scratch)
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            B.sar_rda_form_image(rd.data_ptr(), p, img.data_ptr(), stream.cuda_stream)
+            b.record(stream)
+            torch.cuda.synchronize()
+            if i >= warmup:
+                per.append(a.elapsed_time(b))
+        for s in range(3):
+            for i in range(warmup + steps):
+                flush_l2(torch, scratch)
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(stream)
+                B.sar_rda_run_step(rd.data_ptr(), p, img.data_ptr(), s, stream.cuda_stream)
+                b.record(stream)
+                torch.cuda.synchronize()
+                if i >= warmup:
+                    per_step[s].append(a.elapsed_time(b))
+        B.sar_rda_params_destroy(p)
+        r = summarize(per, metrics.sar_bytes(4096, 4096, dtype), peak)
+        r["ms_per_image"] = r["ms_median"]
+        r["passes_ms"] = {"range_compression": float(np.median(per_step[0])),
+                          "azimuth_fft": float(np.median(per_step[1])),
+                          "rcmc_filter_ifft": float(np.median(per_step[2]))}
+        out[name] = r
+        del ws
+    return out
+
+
+def cpu_baseline(n):
+    """The oracle as it stands, timed on this machine's host cores on a bounded sample."""
+    import oracle
+    sample = 8192
+    x = inputs.gaussian_complex64((sample, n), MAIN["seed"]).astype(np.complex128)
+    oracle.fft_rows(x[:64])
+    t0 = time.perf_counter()
+    oracle.fft_rows(x)
+    dt = time.perf_counter() - t0
+    return {"value": metrics.fft_bytes(n, sample, 0) / dt / 1e9, "unit": "GB/s", "cores": oracle.num_threads(),
+            "kind": "oracle", "seconds": dt,
+            "sample": f"{sample} of 32768 transforms of N={n} (float64 recursive radix-2, OpenMP over transforms)"}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--only-main", dest="only_main", action="store_true",
+                    help="time only the headline workload (skip the other workloads)")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        return run_reference(args)
+    return run_gpu(args)
+
+
+if __name__ == "__main__":
+    sys.exit(main())

@@ -1,0 +1,166 @@
+/*
+ * b200fft — batched complex FFTs and range-Doppler SAR image formation on one
+ * NVIDIA B200 (sm_100a). C ABI: plain pointers and sizes, no C++ or framework
+ * types. Every DEVICE pointer is memory on the current CUDA device, owned by
+ * the caller (for example a torch tensor's data_ptr()); the library allocates
+ * only its own small tables. `stream` is a cudaStream_t passed as void*
+ * (NULL = the default stream). No call synchronises the device unless it says
+ * so; no call falls back to the CPU: what is not supported returns an error.
+ *
+ * Every function returns 0 (B200FFT_OK) or one of the B200FFT_ERR_* codes.
+ */
+#ifndef B200FFT_H
+#define B200FFT_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum {
+    B200FFT_OK = 0,
+    B200FFT_ERR_INVALID_ARG = 1,   /* null pointer, n <= 0, batch <= 0, bad direction or dtype */
+    B200FFT_ERR_UNSUPPORTED = 2,   /* not a power of two, size out of range, layout class */
+    B200FFT_ERR_ALIGNMENT = 3,     /* pointer or stride breaks 128-bit access */
+    B200FFT_ERR_ALLOC = 4,         /* device table allocation failed */
+    B200FFT_ERR_CUDA = 5,          /* launch or runtime error */
+    B200FFT_ERR_WORKSPACE = 6      /* plan needs a workspace that was not set or is too small */
+};
+
+#define B200FFT_FORWARD (-1)       /* exp(-2 pi i n k / N), unnormalised */
+#define B200FFT_INVERSE (+1)       /* exp(+2 pi i n k / N), scaled by 1/N */
+
+#define B200FFT_C64 0              /* interleaved (re, im) fp32, 8 bytes per element */
+#define B200FFT_C32H 1             /* interleaved (re, im) fp16, 4 bytes per element; arithmetic stays fp32 */
+
+typedef struct b200fft_plan_s *fft_plan_t;
+typedef struct b200fft_sar_s *sar_rda_params_t;
+
+/* ------------------------------------------------------------------------
+ * Batched 1-D complex-to-complex transform (paper, Section "The M6 Memory
+ * Hierarchy", the single-pass transform behind Eq. 1: each element is read
+ * from main memory once and written once; Sections "One Pass for N=8192 and
+ * 16384" and "FP16 Storage").
+ *
+ *   forward  X[b][k] =        sum_j x[b][j] exp(-2 pi i j k / n)
+ *   inverse  x[b][j] = (1/n)  sum_k X[b][k] exp(+2 pi i j k / n)
+ *
+ * Element j of transform b lives at index b*dist + j*stride, counted in
+ * complex elements, in the input and in the output alike. Output is in
+ * natural order.
+ *
+ * Supported layouts:
+ *   rows     stride == 1, dist >= n, dist even (dist a multiple of 4 for C32H)
+ *   columns  dist == 1, stride >= batch, stride and batch even: the columns of
+ *            a row-major matrix (paper, Section "End to End": the FFT that
+ *            reads the columns directly)
+ * Supported sizes: n a power of two, 256 <= n <= 16384 in a single pass over
+ * memory; 2^15 <= n <= 2^20 (rows only) by a two-pass four-step split (the
+ * paper's "usual remedy when a transform does not fit on chip"), which needs a
+ * workspace of n*batch elements of the storage type.
+ *
+ * fft_plan_create allocates the plan's twiddle tables on the current device
+ * (at most a few hundred KiB) and builds them there; it synchronises the
+ * device once. The plan may be executed any number of times, on any stream of
+ * that device; concurrent execution on several streams is allowed unless the
+ * plan has a workspace.
+ * ---------------------------------------------------------------------- */
+int fft_plan_create(fft_plan_t *plan, int64_t n, int64_t batch, int64_t stride,
+                    int64_t dist, int direction, int storage_dtype);
+
+/* Bytes of caller-owned DEVICE workspace the plan needs (0 for single-pass plans). */
+int fft_plan_workspace_bytes(fft_plan_t plan, size_t *bytes);
+
+/* Hand the plan a DEVICE workspace (16-byte aligned, at least the size above).
+ * The caller keeps ownership and must keep it alive while the plan executes. */
+int fft_plan_set_workspace(fft_plan_t plan, void *device_ptr, size_t bytes);
+
+/* Enqueue the transform on `stream`. `in` and `out` are DEVICE pointers,
+ * 16-byte aligned, each holding (batch-1)*dist + (n-1)*stride + 1 elements of
+ * the plan's storage type. in == out is allowed; partial overlap is not.
+ * Returns after the launch; B200FFT_ERR_CUDA reports a launch error. */
+int fft_execute(fft_plan_t plan, const void *in, void *out, void *stream);
+
+/* The same transform from HOST buffers (paper's footprint: input plus output):
+ * copies host_in -> dev_in, executes dev_in -> dev_out, copies dev_out ->
+ * host_out, all enqueued on `stream`. The host buffers should be pinned for
+ * the copies to be asynchronous; the device staging buffers are caller-owned
+ * and sized like in/out above. Does not synchronise. */
+int fft_execute_host(fft_plan_t plan, const void *host_in, void *host_out,
+                     void *dev_in, void *dev_out, void *stream);
+
+/* Free the plan's tables. The caller must have synchronised outstanding work. */
+int fft_plan_destroy(fft_plan_t plan);
+
+/* Test knob: force a kernel variant (paper, Section "One Pass": "a regression
+ * test forces N=8192 through this path"). key "four_step" value 1 routes a
+ * rows plan of any supported n >= 4096 through the two-pass split. Unknown
+ * keys return B200FFT_ERR_INVALID_ARG. Must be called before set_workspace. */
+int fft_plan_set_option(fft_plan_t plan, const char *key, int64_t value);
+
+/* Static description of a status code. */
+const char *fft_status_string(int status);
+
+/* Number of kernel launches the library has enqueued since it was loaded
+ * (all plans, all streams); for launch accounting in benchmarks. */
+int64_t b200fft_launch_count(void);
+
+/* ------------------------------------------------------------------------
+ * Range-Doppler SAR image formation (paper, Section "End to End:
+ * Range-Doppler SAR"): range compression (FFT, multiply by the conjugate
+ * chirp spectrum, inverse FFT along each pulse, 1/n_range included); azimuth
+ * FFT along each range bin; range cell migration correction with an 8-tap
+ * sinc interpolator; the azimuth filter exp(+j 4 pi R0 (D - 1) / lambda),
+ * D = sqrt(1 - (lambda f_a / 2 v)^2); azimuth inverse FFT. Three passes over
+ * memory: fused range compression; column FFT; fused RCMC + filter + inverse
+ * column FFT.
+ * ---------------------------------------------------------------------- */
+typedef struct {
+    int64_t n_azimuth;          /* pulses (rows); power of two, 256..16384 */
+    int64_t n_range;            /* range samples per pulse (columns); power of two, 256..16384 */
+    double carrier_hz;
+    double bandwidth_hz;        /* chirp bandwidth; up-chirp, replica centred on t = 0 */
+    double fs_hz;               /* range sampling rate */
+    double pulse_s;             /* pulse length */
+    double prf_hz;
+    double velocity_mps;
+    double r_center_m;          /* slant range of range bin n_range/2 */
+    int32_t intermediate_dtype; /* B200FFT_C64 or B200FFT_C32H for the two intermediate images */
+    int32_t rcmc_taps;          /* must be 8 */
+} sar_rda_desc;
+
+/* Build the processing tables on the current device (conjugate chirp spectrum,
+ * per-Doppler-bin migration and phase coefficients, computed in float64).
+ * Synchronises the device once. */
+int sar_rda_params_create(sar_rda_params_t *params, const sar_rda_desc *desc);
+
+/* Bytes of DEVICE workspace: one intermediate image of n_azimuth*n_range
+ * elements of the intermediate dtype (the azimuth FFT runs in place on it). */
+int sar_rda_workspace_bytes(sar_rda_params_t params, size_t *bytes);
+int sar_rda_set_workspace(sar_rda_params_t params, void *device_ptr, size_t bytes);
+
+/* raw: DEVICE, n_azimuth x n_range interleaved complex fp32, row-major (row =
+ * pulse). out: DEVICE, same shape and type, the focused image; must not alias
+ * raw or the workspace. Enqueues three kernels on `stream`; does not
+ * synchronise. Calls sharing one params object must not overlap on the GPU
+ * (they share its workspace). */
+int sar_rda_form_image(const void *raw, sar_rda_params_t params, void *out, void *stream);
+
+/* Host-buffer variant: copies host_raw -> dev_raw, forms the image into
+ * dev_out, copies dev_out -> host_out, all on `stream`. */
+int sar_rda_form_image_host(const void *host_raw, sar_rda_params_t params, void *host_out,
+                            void *dev_raw, void *dev_out, void *stream);
+
+/* Run one step only, for tests: step 0 range compression (raw -> workspace),
+ * 1 azimuth FFT (workspace, in place), 2 RCMC + filter + inverse FFT
+ * (workspace -> out). `raw` is read by step 0 only, `out` written by step 2 only. */
+int sar_rda_run_step(const void *raw, sar_rda_params_t params, void *out, int step, void *stream);
+
+int sar_rda_params_destroy(sar_rda_params_t params);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* B200FFT_H */

@@ -1,0 +1,27 @@
+// Radix factorisations of the compiled sizes. Cfg<N, W, P, G, r1, r2, r3, r4>:
+// N points, W transforms per tile, P values per thread, G tiles per CTA.
+#pragma once
+#include "fft_core.cuh"
+
+namespace b200fft {
+
+// contiguous rows, one transform per tile
+using R256 = Cfg<256, 1, 32, 16, 16, 16>;
+using R512 = Cfg<512, 1, 32, 8, 16, 2, 16>;
+using R1024 = Cfg<1024, 1, 32, 4, 16, 4, 16>;
+using R2048 = Cfg<2048, 1, 32, 2, 16, 8, 16>;
+using R4096 = Cfg<4096, 1, 32, 1, 16, 16, 16>;
+using R8192 = Cfg<8192, 1, 32, 1, 16, 32, 16>;
+using R16384 = Cfg<16384, 1, 32, 1, 16, 4, 16, 16>;
+
+// W adjacent columns (or rows, in the second pass of the two-pass split) per tile
+using T64 = Cfg<64, 4, 32, 16, 16, 4>;
+using T128 = Cfg<128, 4, 32, 8, 16, 8>;
+using T256 = Cfg<256, 4, 32, 4, 16, 16>;
+using T512 = Cfg<512, 4, 32, 2, 16, 2, 16>;
+using T1024 = Cfg<1024, 4, 32, 1, 16, 4, 16>;
+using T2048 = Cfg<2048, 4, 32, 1, 16, 8, 16>;
+using T4096 = Cfg<4096, 4, 32, 1, 16, 16, 16>;
+using T8192 = Cfg<8192, 2, 32, 1, 16, 32, 16>;
+
+}  // namespace b200fft

@@ -1,0 +1,533 @@
+// Register-resident mixed-radix FFT engine for sm_100a.
+//
+// One "tile" is W transforms of N points that share a CTA's shared memory
+// (W = 1: a contiguous row; W > 1: W adjacent columns of a row-major matrix).
+// Each thread keeps P complex values in registers. The transform is an
+// in-place decimation-in-frequency network N = r1 * r2 * ... * rS: stage s
+// combines, for every other digit fixed, the r_s values whose position differs
+// in digit s (weight L_s = N / (r1..rs)), then multiplies output k by
+// exp(-2 pi i lo k / L_{s-1}) (lo = the lower digits). Between stages the
+// values go through shared memory, each thread writing back exactly the
+// positions it read, so one barrier per exchange is enough. The first stage
+// reads global memory directly in natural order; the last stage leaves
+// X[d1 + r1 d2 + ...] at position (d1, d2, ..) and its threads are assigned
+// with d1 fastest, so the global store is contiguous as well. The same
+// network run backwards (twiddle first, then butterfly, stages S..1) is the
+// decimation-in-time transform that consumes digit-reversed input: used to
+// fuse FFT -> pointwise filter -> inverse FFT without reordering.
+//
+// Shared-memory positions are XOR-swizzled with the top digit so that both the
+// lane-contiguous accesses of stages 1..S-1 and the d1-fastest accesses of the
+// last stage are free of bank conflicts with 128-bit accesses.
+#pragma once
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <cstdint>
+#include <type_traits>
+
+namespace b200fft {
+
+// ---------------------------------------------------------------- utilities
+template <int I>
+using IntC = std::integral_constant<int, I>;
+
+template <int B, int E, class F>
+__device__ __forceinline__ void static_for(F&& f) {
+    if constexpr (B < E) {
+        f(IntC<B>{});
+        static_for<B + 1, E>(f);
+    }
+}
+
+__host__ __device__ constexpr int ilog2(int x) { return x <= 1 ? 0 : 1 + ilog2(x >> 1); }
+
+__device__ __forceinline__ float2 operator+(float2 a, float2 b) { return make_float2(a.x + b.x, a.y + b.y); }
+__device__ __forceinline__ float2 operator-(float2 a, float2 b) { return make_float2(a.x - b.x, a.y - b.y); }
+__device__ __forceinline__ float2 cmul(float2 a, float2 w) {
+    return make_float2(fmaf(a.x, w.x, -a.y * w.y), fmaf(a.x, w.y, a.y * w.x));
+}
+
+// cos / sin of 2 pi m / 32, m = 0..8, as compile-time constants
+__host__ __device__ constexpr double cos32_table(int m) {
+    constexpr double t[9] = {1.0,
+                             0.98078528040323044913,
+                             0.92387953251128675613,
+                             0.83146961230254523708,
+                             0.70710678118654752440,
+                             0.55557023301960222474,
+                             0.38268343236508977173,
+                             0.19509032201612826785,
+                             0.0};
+    return t[m];
+}
+__host__ __device__ constexpr double cos32(int m) {
+    m &= 31;
+    if (m <= 8) return cos32_table(m);
+    if (m <= 16) return -cos32_table(16 - m);
+    if (m <= 24) return -cos32_table(m - 16);
+    return cos32_table(32 - m);
+}
+__host__ __device__ constexpr double sin32(int m) { return cos32(m - 8); }
+
+// x * exp(-2 pi i M / 32), M a compile-time constant
+template <int M_>
+__device__ __forceinline__ float2 mulw32(float2 x) {
+    constexpr int M = M_ & 31;
+    if constexpr (M == 0) return x;
+    else if constexpr (M == 8) return make_float2(x.y, -x.x);
+    else if constexpr (M == 16) return make_float2(-x.x, -x.y);
+    else if constexpr (M == 24) return make_float2(-x.y, x.x);
+    else if constexpr (M == 4) {
+        constexpr float h = 0.70710678118654752440f;
+        return make_float2((x.x + x.y) * h, (x.y - x.x) * h);
+    } else if constexpr (M == 12) {
+        constexpr float h = 0.70710678118654752440f;
+        return make_float2((x.y - x.x) * h, -(x.x + x.y) * h);
+    } else if constexpr (M == 20) {
+        constexpr float h = 0.70710678118654752440f;
+        return make_float2(-(x.x + x.y) * h, (x.x - x.y) * h);
+    } else if constexpr (M == 28) {
+        constexpr float h = 0.70710678118654752440f;
+        return make_float2((x.x - x.y) * h, (x.x + x.y) * h);
+    } else {
+        constexpr float c = (float)cos32(M), s = (float)sin32(M);
+        // (a + ib)(c - is) = (ac + bs) + i(bc - as)
+        return make_float2(fmaf(x.x, c, x.y * s), fmaf(x.y, c, -x.x * s));
+    }
+}
+
+// ------------------------------------------------------- small DFTs in registers
+// Dft<R>::run(v): v[k] <- sum_j v[j] exp(-2 pi i j k / R), natural order in and out.
+template <int R>
+struct Dft;
+
+template <>
+struct Dft<1> {
+    static __device__ __forceinline__ void run(float2*) {}
+};
+template <>
+struct Dft<2> {
+    static __device__ __forceinline__ void run(float2* v) {
+        float2 a = v[0], b = v[1];
+        v[0] = a + b;
+        v[1] = a - b;
+    }
+};
+template <>
+struct Dft<4> {
+    static __device__ __forceinline__ void run(float2* v) {
+        float2 a0 = v[0] + v[2], a1 = v[0] - v[2], a2 = v[1] + v[3], a3 = v[1] - v[3];
+        v[0] = a0 + a2;
+        v[2] = a0 - a2;
+        v[1] = make_float2(a1.x + a3.y, a1.y - a3.x);  // a1 - i a3
+        v[3] = make_float2(a1.x - a3.y, a1.y + a3.x);  // a1 + i a3
+    }
+};
+
+// R = A * B: B-point transforms over j = a + A b, twiddle exp(-2 pi i a c / R),
+// A-point transforms over a; output k = c + B d.
+template <int R, int A, int B>
+__device__ __forceinline__ void dft_composite(float2* v) {
+    float2 y[R];
+    static_for<0, A>([&](auto a_) {
+        constexpr int a = decltype(a_)::value;
+        float2 t[B];
+        static_for<0, B>([&](auto b_) { constexpr int b = decltype(b_)::value; t[b] = v[a + A * b]; });
+        Dft<B>::run(t);
+        static_for<0, B>([&](auto c_) {
+            constexpr int c = decltype(c_)::value;
+            y[a * B + c] = mulw32<a * c * (32 / R)>(t[c]);
+        });
+    });
+    static_for<0, B>([&](auto c_) {
+        constexpr int c = decltype(c_)::value;
+        float2 t[A];
+        static_for<0, A>([&](auto a_) { constexpr int a = decltype(a_)::value; t[a] = y[a * B + c]; });
+        Dft<A>::run(t);
+        static_for<0, A>([&](auto d_) { constexpr int d = decltype(d_)::value; v[c + B * d] = t[d]; });
+    });
+}
+template <>
+struct Dft<8> {
+    static __device__ __forceinline__ void run(float2* v) { dft_composite<8, 2, 4>(v); }
+};
+template <>
+struct Dft<16> {
+    static __device__ __forceinline__ void run(float2* v) { dft_composite<16, 4, 4>(v); }
+};
+template <>
+struct Dft<32> {
+    static __device__ __forceinline__ void run(float2* v) { dft_composite<32, 4, 8>(v); }
+};
+
+// ------------------------------------------------------------ configuration
+template <int N_, int W_, int P_, int G_, int R1_, int R2_, int R3_ = 1, int R4_ = 1>
+struct Cfg {
+    static constexpr int N = N_, W = W_, P = P_, G = G_;
+    static constexpr int S = (R3_ == 1) ? 2 : ((R4_ == 1) ? 3 : 4);
+    __host__ __device__ static constexpr int radix(int s) { return s == 1 ? R1_ : (s == 2 ? R2_ : (s == 3 ? R3_ : R4_)); }
+    __host__ __device__ static constexpr int L(int s) {
+        int l = N;
+        for (int i = 1; i <= s; ++i) l /= radix(i);
+        return l;
+    }
+    static constexpr int T = N * W / P;       // threads per tile
+    static constexpr int THREADS = T * G;     // threads per CTA
+    static constexpr int TILE_ELEMS = N * W;
+    static constexpr int SMEM_BYTES = TILE_ELEMS * G * 8;
+    // twiddle rows of stage s < S start here: (radix-1) rows of L(s) entries each
+    __host__ __device__ static constexpr int tw_off(int s) {
+        int o = 0;
+        for (int i = 1; i < s; ++i) o += (radix(i) - 1) * L(i);
+        return o;
+    }
+    static constexpr int TW_TOTAL = tw_off(S);
+    static_assert(R1_ * R2_ * R3_ * R4_ == N_, "radices must multiply to N");
+    static_assert(L(1) * W_ >= 16, "the swizzle permutes 16-element groups below the top digit");
+    // registers per thread are capped at 128 so that at least 65536 / (128 * THREADS) CTAs fit an SM
+    static constexpr int MINB = (65536 / (128 * THREADS)) > 0 ? (65536 / (128 * THREADS)) : 1;
+    static_assert(P_ % R1_ == 0 && P_ % R2_ == 0 && P_ % R3_ == 0 && P_ % R4_ == 0, "P must be a multiple of every radix");
+    static_assert(P_ / R1_ >= 2 && P_ / radix(S) >= 2, "first and last stage need two butterflies per thread for 128-bit access");
+    static_assert((N_ * W_) % P_ == 0, "tile must divide among threads");
+};
+
+// Geometry of butterfly v of thread t at stage s.
+template <class C, int s>
+struct Geo {
+    static constexpr int r = C::radix(s), V = C::P / r, Ls = C::L(s), Lp = C::L(s - 1), L1 = C::L(1);
+    static constexpr bool last = (s == C::S);
+    static constexpr int W = C::W;
+    static constexpr int estep = last ? W : Ls * W;  // element step per register index j
+    int e0;    // element index (position * W + column) of j = 0, before swizzle
+    int mask;  // swizzle for s > 1
+    int lo;    // twiddle column (stages < S); output index low part (last stage)
+
+    __device__ __forceinline__ void init(int t, int v) {
+        const int c = V * t + v;
+        const int q = c % W;
+        const int b = c / W;
+        if constexpr (!last) {
+            lo = b % Ls;
+            const int hi = b / Ls;
+            const int p0 = hi * Lp + lo;
+            e0 = p0 * W + q;
+            mask = ((p0 / L1) * W) & 14;
+        } else {
+            int rem = b, p0 = 0, d1 = 0;
+            static_for<1, C::S>([&](auto i_) {
+                constexpr int i = decltype(i_)::value;
+                const int d = rem % C::radix(i);
+                rem /= C::radix(i);
+                p0 += d * C::L(i);
+                if constexpr (i == 1) d1 = d;
+            });
+            e0 = p0 * W + q;
+            mask = (d1 * W) & 14;
+            lo = b;
+        }
+    }
+    template <int j>
+    __device__ __forceinline__ int elem() const {
+        if constexpr (s == 1) return (e0 + j * estep) ^ ((j * W) & 14);
+        else return (e0 + j * estep) ^ mask;
+    }
+};
+
+// ------------------------------------------------------------ storage types
+struct StoreC64 {
+    using pair_t = float4;  // two complex fp32
+    static constexpr int ELEM_BYTES = 8;
+    static __device__ __forceinline__ void load2(const void* base, int64_t idx, float2& a, float2& b) {
+        const float4 v = *reinterpret_cast<const float4*>(reinterpret_cast<const float2*>(base) + idx);
+        a = make_float2(v.x, v.y);
+        b = make_float2(v.z, v.w);
+    }
+    static __device__ __forceinline__ void store2(void* base, int64_t idx, float2 a, float2 b) {
+        *reinterpret_cast<float4*>(reinterpret_cast<float2*>(base) + idx) = make_float4(a.x, a.y, b.x, b.y);
+    }
+    static __device__ __forceinline__ float2 load1(const void* base, int64_t idx) {
+        return reinterpret_cast<const float2*>(base)[idx];
+    }
+};
+struct StoreC32H {
+    static constexpr int ELEM_BYTES = 4;
+    static __device__ __forceinline__ void load2(const void* base, int64_t idx, float2& a, float2& b) {
+        const uint2 v = *reinterpret_cast<const uint2*>(reinterpret_cast<const __half2*>(base) + idx);
+        a = __half22float2(*reinterpret_cast<const __half2*>(&v.x));
+        b = __half22float2(*reinterpret_cast<const __half2*>(&v.y));
+    }
+    static __device__ __forceinline__ void store2(void* base, int64_t idx, float2 a, float2 b) {
+        __half2 ha = __float22half2_rn(a), hb = __float22half2_rn(b);
+        uint2 v;
+        v.x = *reinterpret_cast<unsigned*>(&ha);
+        v.y = *reinterpret_cast<unsigned*>(&hb);
+        *reinterpret_cast<uint2*>(reinterpret_cast<__half2*>(base) + idx) = v;
+    }
+    static __device__ __forceinline__ float2 load1(const void* base, int64_t idx) {
+        return __half22float2(reinterpret_cast<const __half2*>(base)[idx]);
+    }
+};
+
+// ------------------------------------------------------------ the engine
+template <class C>
+struct Engine {
+    static constexpr int P = C::P, W = C::W, S = C::S;
+    float2 x[P];
+
+    // ---- shared-memory exchange -------------------------------------------------
+    // Registers of stage s are x[j * V + v]: butterfly v, element j.
+    template <int s, bool WR>
+    __device__ __forceinline__ void smem_rw(float2* sm, int t) {
+        using G = Geo<C, s>;
+        constexpr int V = G::V, r = G::r;
+        if constexpr (G::last && W == 1) {
+            // the two butterflies of a thread sit L1 apart: go 128-bit along j instead
+            static_for<0, V>([&](auto v_) {
+                constexpr int v = decltype(v_)::value;
+                G g;
+                g.init(t, v);
+                static_for<0, r / 2>([&](auto h_) {
+                    constexpr int j = 2 * decltype(h_)::value;
+                    float4* p = reinterpret_cast<float4*>(sm + g.template elem<j>());
+                    if constexpr (WR) {
+                        *p = make_float4(x[j * V + v].x, x[j * V + v].y, x[(j + 1) * V + v].x, x[(j + 1) * V + v].y);
+                    } else {
+                        const float4 q = *p;
+                        x[j * V + v] = make_float2(q.x, q.y);
+                        x[(j + 1) * V + v] = make_float2(q.z, q.w);
+                    }
+                });
+            });
+        } else if constexpr (V >= 2) {
+            static_for<0, V / 2>([&](auto h_) {
+                constexpr int v = 2 * decltype(h_)::value;
+                G g;
+                g.init(t, v);
+                static_for<0, r>([&](auto j_) {
+                    constexpr int j = decltype(j_)::value;
+                    float4* p = reinterpret_cast<float4*>(sm + g.template elem<j>());
+                    if constexpr (WR) {
+                        *p = make_float4(x[j * V + v].x, x[j * V + v].y, x[j * V + v + 1].x, x[j * V + v + 1].y);
+                    } else {
+                        const float4 q = *p;
+                        x[j * V + v] = make_float2(q.x, q.y);
+                        x[j * V + v + 1] = make_float2(q.z, q.w);
+                    }
+                });
+            });
+        } else {
+            G g;
+            g.init(t, 0);
+            static_for<0, r>([&](auto j_) {
+                constexpr int j = decltype(j_)::value;
+                if constexpr (WR) sm[g.template elem<j>()] = x[j];
+                else x[j] = sm[g.template elem<j>()];
+            });
+        }
+    }
+
+    // ---- butterflies + twiddles ----------------------------------------------------
+    // DIT = false: butterfly, then multiply output k by tw[k][lo]   (stages 1..S-1)
+    // DIT = true : multiply input j by tw[j][lo], then butterfly     (transposed network)
+    template <int s, bool DIT>
+    __device__ __forceinline__ void compute(const float2* __restrict__ tw, int t) {
+        using G = Geo<C, s>;
+        constexpr int V = G::V, r = G::r, Ls = G::Ls;
+        constexpr bool has_tw = !G::last;
+        auto twiddle_pair = [&](int lo0, float2* a, float2* b) {
+            // a, b: the r values of butterflies v, v+1 (b == nullptr if V == 1)
+            const float2* row = tw + C::tw_off(s) + lo0;
+            static_for<1, r>([&](auto k_) {
+                constexpr int k = decltype(k_)::value;
+                if constexpr (W == 1 && V >= 2) {
+                    const float4 w = __ldg(reinterpret_cast<const float4*>(row + (k - 1) * Ls));
+                    a[k] = cmul(a[k], make_float2(w.x, w.y));
+                    b[k] = cmul(b[k], make_float2(w.z, w.w));
+                } else {
+                    const float2 w = __ldg(row + (k - 1) * Ls);
+                    a[k] = cmul(a[k], w);
+                    if (b) b[k] = cmul(b[k], w);
+                }
+            });
+        };
+        if constexpr (V >= 2) {
+            static_for<0, V / 2>([&](auto h_) {
+                constexpr int v = 2 * decltype(h_)::value;
+                float2 a[r], b[r];
+                static_for<0, r>([&](auto j_) {
+                    constexpr int j = decltype(j_)::value;
+                    a[j] = x[j * V + v];
+                    b[j] = x[j * V + v + 1];
+                });
+                [[maybe_unused]] int lo0 = 0;
+                if constexpr (has_tw) {
+                    G g;
+                    g.init(t, v);
+                    lo0 = g.lo;
+                    if constexpr (DIT) twiddle_pair(lo0, a, b);
+                }
+                Dft<r>::run(a);
+                Dft<r>::run(b);
+                if constexpr (has_tw && !DIT) twiddle_pair(lo0, a, b);
+                static_for<0, r>([&](auto j_) {
+                    constexpr int j = decltype(j_)::value;
+                    x[j * V + v] = a[j];
+                    x[j * V + v + 1] = b[j];
+                });
+            });
+        } else {
+            [[maybe_unused]] int lo0 = 0;
+            if constexpr (has_tw) {
+                G g;
+                g.init(t, 0);
+                lo0 = g.lo;
+                if constexpr (DIT) twiddle_pair(lo0, x, nullptr);
+            }
+            Dft<r>::run(x);
+            if constexpr (has_tw && !DIT) twiddle_pair(lo0, x, nullptr);
+        }
+    }
+
+    // ---- global access with the stage-1 mapping (natural-order positions) --------------
+    // position of register (j, v): p = j * L1 + lo; rows: index base + p (+1 for v odd);
+    // columns: index base + p * ld + q.
+    template <class ST, bool CONJ>
+    __device__ __forceinline__ void load_first(const void* in, int64_t base, int64_t ld, int t) {
+        using G = Geo<C, 1>;
+        constexpr int V = G::V, r = G::r;
+        static_for<0, V / 2>([&](auto h_) {
+            constexpr int v = 2 * decltype(h_)::value;
+            const int c = V * t + v;
+            const int q = c % W, lo = c / W;
+            static_for<0, r>([&](auto j_) {
+                constexpr int j = decltype(j_)::value;
+                const int64_t idx = (W == 1) ? base + j * G::Ls + lo : base + (int64_t)(j * G::Ls + lo) * ld + q;
+                ST::load2(in, idx, x[j * V + v], x[j * V + v + 1]);
+                if constexpr (CONJ) {
+                    x[j * V + v].y = -x[j * V + v].y;
+                    x[j * V + v + 1].y = -x[j * V + v + 1].y;
+                }
+            });
+        });
+    }
+    template <class ST, bool CONJ>
+    __device__ __forceinline__ void store_first(void* out, int64_t base, int64_t ld, int t, float scale) {
+        using G = Geo<C, 1>;
+        constexpr int V = G::V, r = G::r;
+        static_for<0, V / 2>([&](auto h_) {
+            constexpr int v = 2 * decltype(h_)::value;
+            const int c = V * t + v;
+            const int q = c % W, lo = c / W;
+            static_for<0, r>([&](auto j_) {
+                constexpr int j = decltype(j_)::value;
+                const int64_t idx = (W == 1) ? base + j * G::Ls + lo : base + (int64_t)(j * G::Ls + lo) * ld + q;
+                float2 a = x[j * V + v], b = x[j * V + v + 1];
+                a = make_float2(a.x * scale, (CONJ ? -a.y : a.y) * scale);
+                b = make_float2(b.x * scale, (CONJ ? -b.y : b.y) * scale);
+                ST::store2(out, idx, a, b);
+            });
+        });
+    }
+    // ---- global store with the last-stage mapping: X[lo + (N / r_S) j] ---------------------
+    template <class ST, bool CONJ>
+    __device__ __forceinline__ void store_last(void* out, int64_t base, int64_t ld, int t, float scale) {
+        using G = Geo<C, S>;
+        constexpr int V = G::V, r = G::r;
+        constexpr int KS = C::N / r;
+        static_for<0, V / 2>([&](auto h_) {
+            constexpr int v = 2 * decltype(h_)::value;
+            const int c = V * t + v;
+            const int q = c % W, b0 = c / W;
+            static_for<0, r>([&](auto j_) {
+                constexpr int j = decltype(j_)::value;
+                const int64_t idx = (W == 1) ? base + j * KS + b0 : base + (int64_t)(j * KS + b0) * ld + q;
+                float2 a = x[j * V + v], b = x[j * V + v + 1];
+                a = make_float2(a.x * scale, (CONJ ? -a.y : a.y) * scale);
+                b = make_float2(b.x * scale, (CONJ ? -b.y : b.y) * scale);
+                ST::store2(out, idx, a, b);
+            });
+        });
+    }
+
+    // ---- whole networks ---------------------------------------------------------------
+    // registers hold stage-1 layout on entry; on exit they hold the last stage's
+    // layout: x[j*V + v] = X[b' + (N/r_S) j] for butterfly b' (digit-reversed positions)
+    __device__ __forceinline__ void dif(float2* sm, const float2* __restrict__ tw, int t) {
+        static_for<1, S + 1>([&](auto s_) {
+            constexpr int s = decltype(s_)::value;
+            compute<s, false>(tw, t);
+            if constexpr (s < S) {
+                smem_rw<s, true>(sm, t);
+                __syncthreads();
+                smem_rw<s + 1, false>(sm, t);
+            }
+        });
+    }
+    // registers hold the last stage's layout (digit-reversed positions) on entry,
+    // stage-1 layout in natural order on exit
+    __device__ __forceinline__ void dit(float2* sm, const float2* __restrict__ tw, int t) {
+        static_for<0, S>([&](auto i_) {
+            constexpr int s = S - decltype(i_)::value;
+            compute<s, true>(tw, t);
+            if constexpr (s > 1) {
+                smem_rw<s, true>(sm, t);
+                __syncthreads();
+                smem_rw<s - 1, false>(sm, t);
+            }
+        });
+    }
+};
+
+struct FftArgs {
+    const void* in;
+    void* out;
+    const float2* tw;
+    int64_t tiles;   // rows: batch; columns: batch / W
+    int64_t dist;    // rows: elements between transforms; columns: elements between rows (ld)
+    float scale;
+};
+
+// One CTA = G tiles. INV: inverse via conj(FFT(conj(x))) * scale.
+template <class C, bool INV, class TIn, class TOut>
+__global__ void __launch_bounds__(C::THREADS, C::MINB) fft_kernel(const FftArgs a) {
+    extern __shared__ __align__(16) float2 smem_dyn[];
+    const int g = threadIdx.x / C::T, t = threadIdx.x % C::T;
+    int64_t tile = (int64_t)blockIdx.x * C::G + g;
+    const bool active = tile < a.tiles;
+    if (!active) tile = a.tiles - 1;          // keep the barriers uniform; results discarded
+    float2* sm = smem_dyn + g * C::TILE_ELEMS;
+    const int64_t base = (C::W == 1) ? tile * a.dist : tile * C::W;
+    Engine<C> e;
+    e.template load_first<TIn, INV>(a.in, base, a.dist, t);
+    e.dif(sm, a.tw, t);
+    if (active) e.template store_last<TOut, INV>(a.out, base, a.dist, t, a.scale);
+}
+
+// Builds the per-stage twiddle rows of a configuration in float64, rounds once to fp32:
+// row (k-1) of stage s holds exp(-2 pi i lo k / L_{s-1}), lo = 0 .. L_s - 1.
+template <class C>
+__global__ void build_twiddles_kernel(float2* tw) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= C::TW_TOTAL) return;
+    int s = 1;
+    static_for<1, C::S>([&](auto s_) {
+        constexpr int ss = decltype(s_)::value;
+        if (i >= C::tw_off(ss)) s = ss;
+    });
+    int off = 0, Ls = 1, Lp = 1;
+    static_for<1, C::S>([&](auto s_) {
+        constexpr int ss = decltype(s_)::value;
+        if (s == ss) {
+            off = C::tw_off(ss);
+            Ls = C::L(ss);
+            Lp = C::L(ss - 1);
+        }
+    });
+    const int k = (i - off) / Ls + 1, lo = (i - off) % Ls;
+    const int m = (lo * k) % Lp;                    // exact integer angle index
+    double sn, cs;
+    sincospi(-2.0 * (double)m / (double)Lp, &sn, &cs);
+    tw[i] = make_float2((float)cs, (float)sn);
+}
+
+}  // namespace b200fft

@@ -1,0 +1,19 @@
+// Single-pass batched FFT over contiguous rows: one tile = one transform.
+#include "configs.h"
+#include "registry.h"
+
+namespace b200fft {
+
+static const KernelEntry k_rows[] = {
+    B200FFT_ENTRIES_STD(R256),  B200FFT_ENTRIES_STD(R512),
+    B200FFT_ENTRIES_STD(R1024), B200FFT_ENTRIES_STD(R2048), B200FFT_ENTRIES_STD(R4096),
+    B200FFT_ENTRIES_STD(R8192), B200FFT_ENTRIES_STD(R16384),
+};
+
+const KernelEntry* find_rows_kernel(int n, bool inverse, int in_dtype, int out_dtype) {
+    for (const KernelEntry& e : k_rows)
+        if (e.n == n && e.inverse == inverse && e.in_dtype == in_dtype && e.out_dtype == out_dtype) return &e;
+    return nullptr;
+}
+
+}  // namespace b200fft

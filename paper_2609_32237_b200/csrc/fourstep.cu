@@ -1,0 +1,223 @@
+// Two-pass transform, n = n1 * n2, for n past the on-chip limit (paper, Section
+// "One Pass": the two-pass "four-step" FFT is the usual remedy when a transform
+// does not fit on chip; each extra pass through main memory divides the ceiling).
+//
+// View transform b as an n1 x n2 row-major matrix x[j1][j2].
+//   pass 1: for every column j2, an n1-point transform over j1 (read in place at
+//           stride n2, W adjacent columns per tile), then multiply element
+//           (k1, j2) by exp(-2 pi i j2 k1 / n); written to the workspace as
+//           A[k1][j2].
+//   pass 2: for every row k1 of A, an n2-point transform over j2; X[k1 + n1 k2]
+//           is stored transposed. A tile is W adjacent rows so that the
+//           transposed store writes W*8-byte segments.
+// The inverse conjugates on the way in and on the way out and scales by 1/n.
+#include "../../include/b200fft.h"
+#include "fourstep.h"
+#include "configs.h"
+#include "registry.h"
+
+namespace b200fft {
+
+struct FourStepArgs {
+    const void* in;
+    void* out;
+    const float2* tw;       // stage twiddles of this pass's configuration
+    const float2* tw_lo;
+    const float2* tw_hi;
+    int64_t tiles;          // batch * (columns or rows) / W
+    int64_t groups;         // tiles per transform
+    int64_t dist_in, dist_out;
+    int64_t n, n1, n2;
+    float scale;
+};
+
+struct FourStepEntry {
+    int n, dtype;
+    bool inverse;
+    int w, g, tw_total;
+    cudaError_t (*launch)(const FourStepArgs&, cudaStream_t);
+    cudaError_t (*build_tw)(float2*, cudaStream_t);
+};
+
+template <class C, bool INV, class TIn, class TOut>
+__global__ void __launch_bounds__(C::THREADS, C::MINB) fourstep_pass1_kernel(const FourStepArgs a) {
+    extern __shared__ __align__(16) float2 smem_dyn[];
+    constexpr int W = C::W;
+    const int g = threadIdx.x / C::T, t = threadIdx.x % C::T;
+    int64_t tile = (int64_t)blockIdx.x * C::G + g;
+    const bool active = tile < a.tiles;
+    if (!active) tile = a.tiles - 1;
+    const int64_t b = tile / a.groups, cg = tile % a.groups;
+    float2* sm = smem_dyn + g * C::TILE_ELEMS;
+    Engine<C> e;
+    e.template load_first<TIn, INV>(a.in, b * a.dist_in + cg * W, a.n2, t);
+    e.dif(sm, a.tw, t);
+    if (!active) return;
+    using G = Geo<C, C::S>;
+    constexpr int V = G::V, r = G::r, KS = C::N / r;
+    const int64_t nmask = a.n - 1;
+    static_for<0, V / 2>([&](auto h_) {
+        constexpr int v = 2 * decltype(h_)::value;
+        const int c = V * t + v;
+        const int q = c % W, b0 = c / W;
+        const int64_t j2 = cg * W + q;
+        static_for<0, r>([&](auto j_) {
+            constexpr int j = decltype(j_)::value;
+            const int64_t k1 = j * KS + b0;
+            const int64_t m0 = (k1 * j2) & nmask, m1 = (m0 + k1) & nmask;
+            const float2 w0 = cmul(__ldg(a.tw_hi + (m0 >> 10)), __ldg(a.tw_lo + (m0 & 1023)));
+            const float2 w1 = cmul(__ldg(a.tw_hi + (m1 >> 10)), __ldg(a.tw_lo + (m1 & 1023)));
+            TOut::store2(a.out, b * a.dist_out + k1 * a.n2 + j2, cmul(e.x[j * V + v], w0), cmul(e.x[j * V + v + 1], w1));
+        });
+    });
+}
+
+template <class C, bool INV, class TIn, class TOut>
+__global__ void __launch_bounds__(C::THREADS, C::MINB) fourstep_pass2_kernel(const FourStepArgs a) {
+    extern __shared__ __align__(16) float2 smem_dyn[];
+    constexpr int W = C::W;
+    const int g = threadIdx.x / C::T, t = threadIdx.x % C::T;
+    int64_t tile = (int64_t)blockIdx.x * C::G + g;
+    const bool active = tile < a.tiles;
+    if (!active) tile = a.tiles - 1;
+    const int64_t b = tile / a.groups, rg = tile % a.groups;
+    float2* sm = smem_dyn + g * C::TILE_ELEMS;
+    Engine<C> e;
+    {
+        using G = Geo<C, 1>;
+        constexpr int V = G::V, r = G::r;
+        const int64_t rowbase = b * a.dist_in + rg * W * a.n2;
+        static_for<0, V / 2>([&](auto h_) {
+            constexpr int v = 2 * decltype(h_)::value;
+            const int c = V * t + v;
+            const int q = c % W, lo = c / W;
+            static_for<0, r>([&](auto j_) {
+                constexpr int j = decltype(j_)::value;
+                const int64_t idx = rowbase + (int64_t)q * a.n2 + j * G::Ls + lo;
+                e.x[j * V + v] = TIn::load1(a.in, idx);
+                e.x[j * V + v + 1] = TIn::load1(a.in, idx + a.n2);
+            });
+        });
+    }
+    e.dif(sm, a.tw, t);
+    if (active) e.template store_last<TOut, INV>(a.out, b * a.dist_out + rg * W, a.n1, t, a.scale);
+}
+
+template <class C, bool INV, class TI, class TO, int PASS>
+cudaError_t launch_fourstep(const FourStepArgs& a, cudaStream_t st) {
+    static bool done[64] = {};
+    auto kernel = (PASS == 1) ? fourstep_pass1_kernel<C, INV, TI, TO> : fourstep_pass2_kernel<C, INV, TI, TO>;
+    cudaError_t e = ensure_smem(kernel, C::SMEM_BYTES, done);
+    if (e != cudaSuccess) return e;
+    const int64_t grid = (a.tiles + C::G - 1) / C::G;
+    kernel<<<(unsigned)grid, C::THREADS, C::SMEM_BYTES, st>>>(a);
+    g_launch_count.fetch_add(1, std::memory_order_relaxed);
+    return cudaGetLastError();
+}
+
+template <class C, bool INV, class TS, int PASS>
+constexpr FourStepEntry make_fs_entry() {
+    return FourStepEntry{C::N, TS::ELEM_BYTES == 8 ? 0 : 1, INV, C::W, C::G, C::TW_TOTAL,
+                         &launch_fourstep<C, INV, TS, TS, PASS>, &launch_build_tw<C>};
+}
+#define FS_ENTRIES(C, PASS)                                                         \
+    make_fs_entry<C, false, StoreC64, PASS>(), make_fs_entry<C, true, StoreC64, PASS>(), \
+    make_fs_entry<C, false, StoreC32H, PASS>(), make_fs_entry<C, true, StoreC32H, PASS>()
+
+static const FourStepEntry k_pass1[] = {FS_ENTRIES(T64, 1), FS_ENTRIES(T128, 1), FS_ENTRIES(T256, 1),
+                                        FS_ENTRIES(T512, 1), FS_ENTRIES(T1024, 1)};
+static const FourStepEntry k_pass2[] = {FS_ENTRIES(T64, 2), FS_ENTRIES(T128, 2), FS_ENTRIES(T256, 2),
+                                        FS_ENTRIES(T512, 2), FS_ENTRIES(T1024, 2)};
+
+template <size_t K>
+static const FourStepEntry* find(const FourStepEntry (&tab)[K], int n, bool inv, int dtype) {
+    for (const FourStepEntry& e : tab)
+        if (e.n == n && e.inverse == inv && e.dtype == dtype) return &e;
+    return nullptr;
+}
+
+// exp(-2 pi i m step / n) for m = 0..count-1, float64 then one rounding
+__global__ void build_factor_table(float2* tab, int count, int64_t step, int64_t n) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= count) return;
+    const int64_t m = ((int64_t)i * step) % n;
+    double sn, cs;
+    sincospi(-2.0 * (double)m / (double)n, &sn, &cs);
+    tab[i] = make_float2((float)cs, (float)sn);
+}
+
+void fourstep_release(FourStep* fs) {
+    if (fs->tw1) cudaFree(fs->tw1);
+    if (fs->tw2) cudaFree(fs->tw2);
+    if (fs->tw_lo) cudaFree(fs->tw_lo);
+    if (fs->tw_hi) cudaFree(fs->tw_hi);
+    *fs = FourStep();
+}
+
+int fourstep_build(FourStep* fs, int64_t n, int64_t batch, int64_t dist, int direction, int dtype) {
+    fourstep_release(fs);
+    int lg = 0;
+    while (((int64_t)1 << lg) < n) ++lg;
+    if (((int64_t)1 << lg) != n || lg < 12 || lg > 20) return B200FFT_ERR_UNSUPPORTED;
+    fs->n = n;
+    fs->n1 = (int64_t)1 << ((lg + 1) / 2);
+    fs->n2 = n / fs->n1;
+    fs->batch = batch;
+    fs->dist = dist;
+    fs->direction = direction;
+    fs->dtype = dtype;
+    const bool inv = direction == B200FFT_INVERSE;
+    fs->pass1 = find(k_pass1, (int)fs->n1, inv, dtype);
+    fs->pass2 = find(k_pass2, (int)fs->n2, inv, dtype);
+    if (!fs->pass1 || !fs->pass2) return B200FFT_ERR_UNSUPPORTED;
+    const int hi_count = (int)(n / 1024);
+    if (cudaMalloc(&fs->tw1, sizeof(float2) * (size_t)fs->pass1->tw_total) != cudaSuccess ||
+        cudaMalloc(&fs->tw2, sizeof(float2) * (size_t)fs->pass2->tw_total) != cudaSuccess ||
+        cudaMalloc(&fs->tw_lo, sizeof(float2) * 1024) != cudaSuccess ||
+        cudaMalloc(&fs->tw_hi, sizeof(float2) * (size_t)hi_count) != cudaSuccess) {
+        cudaGetLastError();
+        fourstep_release(fs);
+        return B200FFT_ERR_ALLOC;
+    }
+    bool ok = fs->pass1->build_tw(fs->tw1, 0) == cudaSuccess && fs->pass2->build_tw(fs->tw2, 0) == cudaSuccess;
+    build_factor_table<<<4, 256>>>(fs->tw_lo, 1024, 1, n);
+    build_factor_table<<<(hi_count + 255) / 256, 256>>>(fs->tw_hi, hi_count, 1024, n);
+    g_launch_count.fetch_add(2, std::memory_order_relaxed);
+    ok = ok && cudaGetLastError() == cudaSuccess && cudaStreamSynchronize(0) == cudaSuccess;
+    if (!ok) {
+        fourstep_release(fs);
+        return B200FFT_ERR_CUDA;
+    }
+    return B200FFT_OK;
+}
+
+int fourstep_execute(const FourStep* fs, const void* in, void* out, void* workspace, cudaStream_t st) {
+    FourStepArgs a;
+    a.tw_lo = fs->tw_lo;
+    a.tw_hi = fs->tw_hi;
+    a.n = fs->n;
+    a.n1 = fs->n1;
+    a.n2 = fs->n2;
+    a.scale = (fs->direction == B200FFT_INVERSE) ? (float)(1.0 / (double)fs->n) : 1.0f;
+    // pass 1: columns of every n1 x n2 matrix
+    a.in = in;
+    a.out = workspace;
+    a.tw = fs->tw1;
+    a.groups = fs->n2 / fs->pass1->w;
+    a.tiles = fs->batch * a.groups;
+    a.dist_in = fs->dist;
+    a.dist_out = fs->n;
+    if (fs->pass1->launch(a, st) != cudaSuccess) return B200FFT_ERR_CUDA;
+    // pass 2: rows of the workspace, transposed store
+    a.in = workspace;
+    a.out = out;
+    a.tw = fs->tw2;
+    a.groups = fs->n1 / fs->pass2->w;
+    a.tiles = fs->batch * a.groups;
+    a.dist_in = fs->n;
+    a.dist_out = fs->dist;
+    if (fs->pass2->launch(a, st) != cudaSuccess) return B200FFT_ERR_CUDA;
+    return B200FFT_OK;
+}
+
+}  // namespace b200fft

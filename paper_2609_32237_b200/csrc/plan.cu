@@ -1,0 +1,196 @@
+// C ABI of the FFT plans: argument validation, variant choice, table ownership.
+#include <cuda_runtime.h>
+#include <cstring>
+#include <new>
+#include "../../include/b200fft.h"
+#include "registry.h"
+#include "fourstep.h"
+
+namespace b200fft {
+std::atomic<int64_t> g_launch_count{0};
+}
+
+using namespace b200fft;
+
+enum Layout { LAYOUT_ROWS = 0, LAYOUT_COLS = 1 };
+
+struct b200fft_plan_s {
+    int64_t n, batch, stride, dist;
+    int direction, dtype;
+    Layout layout;
+    bool four_step;
+    const KernelEntry* kernel;   // single-pass variant
+    float2* tw;                  // its twiddle rows (device)
+    int device;
+    FourStep fs;                 // two-pass variant
+    void* workspace;
+    size_t workspace_bytes;
+};
+
+static bool is_pow2(int64_t v) { return v > 0 && (v & (v - 1)) == 0; }
+
+static int elem_bytes(int dtype) { return dtype == B200FFT_C64 ? 8 : 4; }
+
+static int build_single_pass(b200fft_plan_s* p) {
+    const bool inv = p->direction == B200FFT_INVERSE;
+    p->kernel = (p->layout == LAYOUT_ROWS) ? find_rows_kernel((int)p->n, inv, p->dtype, p->dtype)
+                                           : find_cols_kernel((int)p->n, inv, p->dtype, p->dtype);
+    if (!p->kernel) return B200FFT_ERR_UNSUPPORTED;
+    if (cudaMalloc(&p->tw, sizeof(float2) * (size_t)p->kernel->tw_total) != cudaSuccess) {
+        cudaGetLastError();
+        return B200FFT_ERR_ALLOC;
+    }
+    if (p->kernel->build_tw(p->tw, 0) != cudaSuccess) return B200FFT_ERR_CUDA;
+    if (cudaStreamSynchronize(0) != cudaSuccess) return B200FFT_ERR_CUDA;
+    return B200FFT_OK;
+}
+
+static void release(b200fft_plan_s* p) {
+    if (p->tw) cudaFree(p->tw);
+    p->tw = nullptr;
+    fourstep_release(&p->fs);
+}
+
+extern "C" int fft_plan_create(fft_plan_t* plan, int64_t n, int64_t batch, int64_t stride,
+                               int64_t dist, int direction, int storage_dtype) {
+    if (!plan) return B200FFT_ERR_INVALID_ARG;
+    *plan = nullptr;
+    if (n <= 0 || batch <= 0 || stride <= 0 || dist <= 0) return B200FFT_ERR_INVALID_ARG;
+    if (direction != B200FFT_FORWARD && direction != B200FFT_INVERSE) return B200FFT_ERR_INVALID_ARG;
+    if (storage_dtype != B200FFT_C64 && storage_dtype != B200FFT_C32H) return B200FFT_ERR_INVALID_ARG;
+    if (!is_pow2(n)) return B200FFT_ERR_UNSUPPORTED;
+    if (n < 256 || n > (1 << 20)) return B200FFT_ERR_UNSUPPORTED;
+
+    Layout layout;
+    if (stride == 1 && dist >= n) layout = LAYOUT_ROWS;
+    else if (dist == 1 && stride >= batch) layout = LAYOUT_COLS;
+    else return B200FFT_ERR_UNSUPPORTED;
+    // 128-bit (c64) or 64-bit (c32h) vector access: two elements at a time
+    const int64_t align_elems = (storage_dtype == B200FFT_C64) ? 2 : 4;
+    if (layout == LAYOUT_ROWS && dist % align_elems) return B200FFT_ERR_ALIGNMENT;
+    if (layout == LAYOUT_COLS && (stride % align_elems || batch % 2)) return B200FFT_ERR_ALIGNMENT;
+
+    b200fft_plan_s* p = new (std::nothrow) b200fft_plan_s();
+    if (!p) return B200FFT_ERR_ALLOC;
+    p->n = n; p->batch = batch; p->stride = stride; p->dist = dist;
+    p->direction = direction; p->dtype = storage_dtype; p->layout = layout;
+    if (cudaGetDevice(&p->device) != cudaSuccess) { delete p; return B200FFT_ERR_CUDA; }
+
+    int rc;
+    if (n > 16384) {
+        if (layout != LAYOUT_ROWS) { delete p; return B200FFT_ERR_UNSUPPORTED; }
+        p->four_step = true;
+        rc = fourstep_build(&p->fs, n, batch, dist, direction, storage_dtype);
+    } else {
+        if (layout == LAYOUT_COLS) {
+            const KernelEntry* k = find_cols_kernel((int)n, false, storage_dtype, storage_dtype);
+            if (!k) { delete p; return B200FFT_ERR_UNSUPPORTED; }
+            if (batch % k->w) { delete p; return B200FFT_ERR_UNSUPPORTED; }
+        }
+        rc = build_single_pass(p);
+    }
+    if (rc != B200FFT_OK) { release(p); delete p; return rc; }
+    *plan = p;
+    return B200FFT_OK;
+}
+
+extern "C" int fft_plan_set_option(fft_plan_t p, const char* key, int64_t value) {
+    if (!p || !key) return B200FFT_ERR_INVALID_ARG;
+    if (std::strcmp(key, "four_step") == 0) {
+        if (p->layout != LAYOUT_ROWS || p->n < 4096) return B200FFT_ERR_UNSUPPORTED;
+        if (value && !p->four_step) {
+            int rc = fourstep_build(&p->fs, p->n, p->batch, p->dist, p->direction, p->dtype);
+            if (rc != B200FFT_OK) return rc;
+            p->four_step = true;
+            p->workspace = nullptr;
+            p->workspace_bytes = 0;
+        } else if (!value && p->four_step && p->n <= 16384) {
+            if (!p->kernel) {
+                int rc = build_single_pass(p);
+                if (rc != B200FFT_OK) return rc;
+            }
+            p->four_step = false;
+        }
+        return B200FFT_OK;
+    }
+    return B200FFT_ERR_INVALID_ARG;
+}
+
+extern "C" int fft_plan_workspace_bytes(fft_plan_t p, size_t* bytes) {
+    if (!p || !bytes) return B200FFT_ERR_INVALID_ARG;
+    *bytes = p->four_step ? (size_t)p->n * (size_t)p->batch * (size_t)elem_bytes(p->dtype) : 0;
+    return B200FFT_OK;
+}
+
+extern "C" int fft_plan_set_workspace(fft_plan_t p, void* ptr, size_t bytes) {
+    if (!p) return B200FFT_ERR_INVALID_ARG;
+    size_t need = 0;
+    fft_plan_workspace_bytes(p, &need);
+    if (need == 0) { p->workspace = ptr; p->workspace_bytes = bytes; return B200FFT_OK; }
+    if (!ptr) return B200FFT_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(ptr) % 16) return B200FFT_ERR_ALIGNMENT;
+    if (bytes < need) return B200FFT_ERR_WORKSPACE;
+    p->workspace = ptr;
+    p->workspace_bytes = bytes;
+    return B200FFT_OK;
+}
+
+extern "C" int fft_execute(fft_plan_t p, const void* in, void* out, void* stream) {
+    if (!p || !in || !out) return B200FFT_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(in) % 16 || reinterpret_cast<uintptr_t>(out) % 16) return B200FFT_ERR_ALIGNMENT;
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    if (p->four_step) {
+        size_t need = 0;
+        fft_plan_workspace_bytes(p, &need);
+        if (!p->workspace || p->workspace_bytes < need) return B200FFT_ERR_WORKSPACE;
+        return fourstep_execute(&p->fs, in, out, p->workspace, st);
+    }
+    FftArgs a;
+    a.in = in;
+    a.out = out;
+    a.tw = p->tw;
+    a.scale = (p->direction == B200FFT_INVERSE) ? (float)(1.0 / (double)p->n) : 1.0f;
+    if (p->layout == LAYOUT_ROWS) {
+        a.tiles = p->batch;
+        a.dist = p->dist;
+    } else {
+        a.tiles = p->batch / p->kernel->w;
+        a.dist = p->stride;
+    }
+    return p->kernel->launch(a, st) == cudaSuccess ? B200FFT_OK : B200FFT_ERR_CUDA;
+}
+
+extern "C" int fft_execute_host(fft_plan_t p, const void* host_in, void* host_out,
+                                void* dev_in, void* dev_out, void* stream) {
+    if (!p || !host_in || !host_out || !dev_in || !dev_out) return B200FFT_ERR_INVALID_ARG;
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    const size_t elems = (size_t)((p->batch - 1) * p->dist + (p->n - 1) * p->stride + 1);
+    const size_t bytes = elems * (size_t)elem_bytes(p->dtype);
+    if (cudaMemcpyAsync(dev_in, host_in, bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return B200FFT_ERR_CUDA;
+    int rc = fft_execute(p, dev_in, dev_out, stream);
+    if (rc != B200FFT_OK) return rc;
+    if (cudaMemcpyAsync(host_out, dev_out, bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess) return B200FFT_ERR_CUDA;
+    return B200FFT_OK;
+}
+
+extern "C" int fft_plan_destroy(fft_plan_t p) {
+    if (!p) return B200FFT_ERR_INVALID_ARG;
+    release(p);
+    delete p;
+    return B200FFT_OK;
+}
+
+extern "C" const char* fft_status_string(int status) {
+    switch (status) {
+    case B200FFT_OK: return "ok";
+    case B200FFT_ERR_INVALID_ARG: return "invalid argument";
+    case B200FFT_ERR_UNSUPPORTED: return "unsupported size or layout";
+    case B200FFT_ERR_ALIGNMENT: return "pointer or stride not aligned for vector access";
+    case B200FFT_ERR_ALLOC: return "allocation failed";
+    case B200FFT_ERR_CUDA: return "CUDA runtime or launch error";
+    case B200FFT_ERR_WORKSPACE: return "workspace missing or too small";
+    default: return "unknown status";
+    }
+}
+
+extern "C" int64_t b200fft_launch_count(void) { return g_launch_count.load(); }

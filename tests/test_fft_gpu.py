@@ -1,0 +1,242 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the float64
+oracle on the same seeded inputs. Tolerances: relative L2 <= 1e-5 for fp32
+storage, <= 5e-3 for fp16 storage (worst single transform and pooled)."""
+import numpy as np
+import pytest
+
+import oracle
+from paper_2609_32237_b200 import inputs
+from gpu_util import (have_gpu, rel_l2, worst_rel_l2, to_device_c64, to_device_half, run_fft, half_to_c128)
+
+pytestmark = pytest.mark.gpu
+
+TOL32 = 1e-5
+TOL16 = 5e-3
+FWD, INV = -1, 1
+C64, C32H = 0, 1
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _need_gpu():
+    if not have_gpu():
+        pytest.skip("no CUDA device")
+
+
+def _check_rows(n, batch, seed, dist=None, gaussian=False, direction=FWD, options=None, tol=TOL32):
+    dist = dist or n
+    gen = inputs.gaussian_complex64 if gaussian else inputs.uniform_complex64
+    buf = gen((batch, dist), seed)
+    x = buf[:, :n]
+    want = oracle.fft_rows(x.astype(np.complex128), direction)
+    got = run_fft(to_device_c64(buf), n, batch, 1, dist, direction, C64, options=options).cpu().numpy()
+    worst, pooled = worst_rel_l2(got[:, :n], want)
+    assert worst <= tol and pooled <= tol, (n, batch, worst, pooled)
+    if dist > n:   # padding between transforms must stay untouched (output buffer was zero-filled)
+        assert np.all(got[:, n:] == 0)
+    return worst
+
+
+def test_config0_whole_batch_and_round_trip():
+    """N = 1024, batch 256, uniform [-1, 1), seed 0: every transform against the direct DFT."""
+    x = inputs.uniform_complex64((256, 1024), 0)
+    want = oracle.fft_rows(x.astype(np.complex128), FWD)
+    xd = to_device_c64(x)
+    y = run_fft(xd, 1024, 256, 1, 1024, FWD, C64)
+    worst, pooled = worst_rel_l2(y.cpu().numpy(), want)
+    assert worst <= TOL32 and pooled <= TOL32
+    back = run_fft(y, 1024, 256, 1, 1024, INV, C64).cpu().numpy()
+    assert rel_l2(back, x) <= TOL32
+    want_inv = oracle.fft_rows(x.astype(np.complex128), INV)
+    got_inv = run_fft(xd, 1024, 256, 1, 1024, INV, C64).cpu().numpy()
+    assert max(worst_rel_l2(got_inv, want_inv)) <= TOL32
+
+
+@pytest.mark.parametrize("n", [256, 512, 1024, 2048, 4096, 8192, 16384])
+@pytest.mark.parametrize("direction", [FWD, INV])
+def test_rows_every_size_ragged_batch(n, direction):
+    # batches that do not fill the last CTA of multi-transform configurations
+    for batch in (1, 5, 37):
+        _check_rows(n, batch, seed=100 + n % 97 + batch, direction=direction, gaussian=(batch == 37))
+
+
+def test_rows_with_padding_between_transforms():
+    _check_rows(4096, 9, seed=7, dist=4096 + 6)
+    _check_rows(1024, 11, seed=8, dist=1024 + 2)
+
+
+def test_rows_closed_forms_on_gpu():
+    n = 8192
+    x = np.zeros((3, n), dtype=np.complex64)
+    x[0, 0] = 1                                  # impulse -> ones
+    x[1, :] = 1                                  # ones -> n * delta
+    x[2, :] = np.exp(2j * np.pi * 77 * np.arange(n) / n)   # tone -> n * delta at 77
+    y = run_fft(to_device_c64(x), n, 3, 1, n, FWD, C64).cpu().numpy()
+    assert np.abs(y[0] - 1).max() < 1e-6
+    e = np.zeros(n); e[0] = n
+    assert np.abs(y[1] - e).max() < 1e-2
+    e = np.zeros(n); e[77] = n
+    assert np.abs(y[2] - e).max() < 0.2 and abs(y[2, 77] - n) < 0.05
+
+
+def test_rows_in_place_and_deterministic():
+    x = inputs.gaussian_complex64((6, 4096), 21)
+    a = run_fft(to_device_c64(x), 4096, 6, 1, 4096, FWD, C64).cpu().numpy()
+    b = run_fft(to_device_c64(x), 4096, 6, 1, 4096, FWD, C64, inplace=True).cpu().numpy()
+    c = run_fft(to_device_c64(x), 4096, 6, 1, 4096, FWD, C64).cpu().numpy()
+    assert np.array_equal(a.view(np.uint64), b.view(np.uint64))
+    assert np.array_equal(a.view(np.uint64), c.view(np.uint64))
+
+
+@pytest.mark.parametrize("n", [1024, 4096, 8192, 16384])
+@pytest.mark.parametrize("direction", [FWD, INV])
+def test_rows_fp16_storage(n, direction):
+    batch = 6
+    x = inputs.gaussian_complex64((batch, n), 2)
+    if direction == INV:
+        x = x * np.float32(8.0)
+    h = inputs.to_half_storage(x)
+    want = oracle.fft_rows(inputs.from_half_storage(h), direction)   # oracle sees the fp16-rounded input
+    got = half_to_c128(run_fft(to_device_half(h), n, batch, 1, n, direction, C32H))
+    worst, pooled = worst_rel_l2(got, want)
+    assert worst <= TOL16 and pooled <= TOL16
+    assert -20 * np.log10(pooled) > 60.0       # fp32 exchange: well above the gate (paper: ~73.6 dB)
+
+
+@pytest.mark.parametrize("n,cols,ld", [(256, 8, 8), (512, 12, 16), (1024, 20, 20), (2048, 8, 10),
+                                       (4096, 12, 12), (8192, 6, 6)])
+@pytest.mark.parametrize("direction", [FWD, INV])
+def test_columns(n, cols, ld, direction):
+    m = inputs.uniform_complex64((n, ld), 3)
+    want = oracle.fft_cols(m[:, :cols].astype(np.complex128), direction)
+    got = run_fft(to_device_c64(m), n, cols, ld, 1, direction, C64).cpu().numpy()
+    assert rel_l2(got[:, :cols], want) <= TOL32
+    per_col = np.linalg.norm(got[:, :cols] - want, axis=0) / np.linalg.norm(want, axis=0)
+    assert per_col.max() <= TOL32
+    if ld > cols:
+        assert np.all(got[:, cols:] == 0)
+
+
+def test_columns_fp16_and_in_place():
+    n, cols = 4096, 8
+    m = inputs.uniform_complex64((n, cols), 31)
+    h = inputs.to_half_storage(m)
+    want = oracle.fft_cols(inputs.from_half_storage(h), FWD)
+    got = half_to_c128(run_fft(to_device_half(h), n, cols, cols, 1, FWD, C32H, inplace=True))
+    assert rel_l2(got, want) <= TOL16
+
+
+def test_2d_small():
+    m = inputs.uniform_complex64((512, 256), 32)
+    want = oracle.fft2d(m.astype(np.complex128))
+    d = to_device_c64(m)
+    d = run_fft(d, 256, 512, 1, 256, FWD, C64, inplace=True)
+    d = run_fft(d, 512, 256, 256, 1, FWD, C64, inplace=True)
+    assert rel_l2(d.cpu().numpy(), want) <= TOL32
+
+
+def test_config3_columns_and_2d_full():
+    """4096 x 4096 row-major, uniform [-1, 1), seed 3: all columns, then the full 2-D transform."""
+    m = inputs.uniform_complex64((4096, 4096), 3)
+    want_cols = oracle.fft_cols(m.astype(np.complex128), FWD)
+    d = to_device_c64(m)
+    got = run_fft(d, 4096, 4096, 4096, 1, FWD, C64).cpu().numpy()
+    per_col = np.linalg.norm(got - want_cols, axis=0) / np.linalg.norm(want_cols, axis=0)
+    assert per_col.max() <= TOL32 and rel_l2(got, want_cols) <= TOL32
+    del want_cols
+    want2d = oracle.fft2d(m.astype(np.complex128))
+    d = run_fft(d, 4096, 4096, 1, 4096, FWD, C64, inplace=True)
+    d = run_fft(d, 4096, 4096, 4096, 1, FWD, C64, inplace=True)
+    assert rel_l2(d.cpu().numpy(), want2d) <= TOL32
+
+
+@pytest.mark.parametrize("n", [4096, 8192, 16384])
+@pytest.mark.parametrize("direction", [FWD, INV])
+def test_four_step_forced_at_single_pass_sizes(n, direction):
+    """The two-pass split forced at sizes the single-pass kernels also cover
+    (the paper's regression-test idea): whole batch against the oracle."""
+    _check_rows(n, 5, seed=41, direction=direction, options={"four_step": 1})
+
+
+@pytest.mark.parametrize("lg", [15, 16, 17, 18, 20])
+def test_four_step_large(lg):
+    n = 1 << lg
+    batch = 3 if lg < 20 else 2
+    _check_rows(n, batch, seed=50 + lg, gaussian=True)
+    _check_rows(n, batch, seed=60 + lg, direction=INV)
+
+
+def test_four_step_fp16_and_workspace_errors():
+    import torch
+    from paper_2609_32237_b200 import binding as B
+    n, batch = 1 << 16, 2
+    x = inputs.gaussian_complex64((batch, n), 71)
+    h = inputs.to_half_storage(x)
+    want = oracle.fft_rows(inputs.from_half_storage(h), FWD)
+    got = half_to_c128(run_fft(to_device_half(h), n, batch, 1, n, FWD, C32H))
+    assert max(worst_rel_l2(got, want)) <= TOL16
+    plan = B.fft_plan_create(n, batch, 1, n, FWD, C64)
+    try:
+        need = B.fft_plan_workspace_bytes(plan)
+        assert need == n * batch * 8
+        d = to_device_c64(x)
+        with pytest.raises(B.B200FftError) as e:
+            B.fft_execute(plan, d.data_ptr(), d.data_ptr(), 0)
+        assert e.value.status == 6
+        small = torch.empty(need // 2, dtype=torch.uint8, device="cuda")
+        with pytest.raises(B.B200FftError) as e:
+            B.fft_plan_set_workspace(plan, small.data_ptr(), need // 2)
+        assert e.value.status == 6
+        with pytest.raises(B.B200FftError) as e:
+            B.fft_execute(plan, d.data_ptr() + 8, d.data_ptr(), 0)
+        assert e.value.status == 3
+    finally:
+        B.fft_plan_destroy(plan)
+
+
+def _sampled_full_size(n, batch, seed, dtype, direction=FWD):
+    """Full-size batch in the launch configuration the bench times: 64 sampled
+    transforms against the oracle, plus two whole-batch invariants computed
+    outside the library (Parseval and the DC bin)."""
+    import torch
+    x = inputs.gaussian_complex64((batch, n), seed)
+    idx = inputs.sample_indices(batch, 64, seed)
+    if dtype == C64:
+        xd = to_device_c64(x)
+        y = run_fft(xd, n, batch, 1, n, direction, C64)
+        got = y[torch.from_numpy(idx).cuda()].cpu().numpy()
+        want = oracle.fft_rows(x[idx].astype(np.complex128), direction)
+        tol = TOL32
+        yc, xc = y, xd
+    else:
+        h = inputs.to_half_storage(x)
+        del x
+        hd = to_device_half(h)
+        y = run_fft(hd, n, batch, 1, n, direction, C32H)
+        got = half_to_c128(y[torch.from_numpy(idx).cuda()])
+        want = oracle.fft_rows(inputs.from_half_storage(h[idx]), direction)
+        tol = TOL16
+        yc = torch.view_as_complex(y.float())
+        xc = torch.view_as_complex(hd.float())
+    worst, pooled = worst_rel_l2(got, want)
+    assert worst <= tol and pooled <= tol, (worst, pooled)
+    if direction == FWD:
+        ex = (xc.abs().double() ** 2).sum(-1)
+        ey = (yc.abs().double() ** 2).sum(-1)
+        assert float(((ey - n * ex).abs() / (n * ex)).max()) <= (1e-5 if dtype == C64 else 5e-3)
+        dc = xc.to(torch.complex128).sum(-1)
+        scale = float(n) ** 0.5 * 2.0
+        assert float((yc[:, 0].to(torch.complex128) - dc).abs().max()) <= (1e-4 if dtype == C64 else 0.2) * scale
+    return pooled
+
+
+def test_config1_full_size_forward_and_inverse():
+    """N = 4096, batch 32768 (1 GiB), Gaussian sigma = 1, seed 1."""
+    _sampled_full_size(4096, 32768, 1, C64, FWD)
+    _sampled_full_size(4096, 32768, 1, C64, INV)
+
+
+@pytest.mark.parametrize("n,batch", [(8192, 16384), (16384, 8192)])
+@pytest.mark.parametrize("dtype", [C64, C32H])
+def test_config2_full_size(n, batch, dtype):
+    """N = 8192 x 16384 and N = 16384 x 8192, Gaussian, seed 2, fp32 and fp16 storage."""
+    _sampled_full_size(n, batch, 2, dtype, FWD)

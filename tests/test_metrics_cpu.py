@@ -1,0 +1,27 @@
+"""The throughput arithmetic used by the bench, pinned to the numbers the paper prints."""
+from paper_2609_32237_b200 import metrics
+from conftest import read_golden
+
+
+def test_eq1_ceilings_match_the_paper():
+    g = read_golden("paper_eq1_ceilings.txt")
+    bw = g["bandwidth_gbs"]
+    for n in (4096, 8192, 16384):
+        assert abs(metrics.single_pass_ceiling_gflops(n, bw, 0) - g[f"fp32_gflops_{n}"]) <= 0.6
+        assert abs(metrics.single_pass_ceiling_gflops(n, bw, 1) - g[f"fp16_gflops_{n}"]) <= 1.0
+
+
+def test_gflops_and_effective_bandwidth_are_consistent_with_the_paper_row():
+    g = read_golden("paper_eq1_ceilings.txt")
+    assert abs(metrics.gflops_to_gbs(g["row_gflops"], 4096, 0) - g["row_gbs"]) <= 1.0
+    # a batch timed at exactly the ceiling reports the bandwidth it was derived from
+    n, b = 8192, 2048
+    secs = metrics.fft_bytes(n, b, 0) / (150e9)
+    assert abs(metrics.fft_gflops(n, b, secs) - metrics.single_pass_ceiling_gflops(n, 150.0)) < 1e-6
+
+
+def test_footprints():
+    assert metrics.fft_bytes(4096, 32768, 0) == 2 * 1024 ** 3      # 1 GiB in + 1 GiB out
+    assert metrics.fft_bytes(8192, 16384, 1) == 1024 ** 3
+    assert metrics.sar_bytes(4096, 4096, 0) == 48 * 4096 * 4096
+    assert metrics.sar_bytes(4096, 4096, 1) == 32 * 4096 * 4096

@@ -1,0 +1,126 @@
+"""GPU parity of the range-Doppler chain against the float64 oracle: each
+pass on its own, the whole image (relative L2 <= 1e-5 with fp32
+intermediates, <= 5e-3 with fp16), and every target's peak cell exactly."""
+import numpy as np
+import pytest
+
+import oracle
+from oracle import quality
+from paper_2609_32237_b200 import inputs
+from gpu_util import have_gpu, rel_l2, to_device_c64, half_to_c128
+
+pytestmark = pytest.mark.gpu
+C64, C32H = 0, 1
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _need_gpu():
+    if not have_gpu():
+        pytest.skip("no CUDA device")
+
+
+def _gpu_chain(scene, raw, dtype, steps=False):
+    import torch
+    from paper_2609_32237_b200 import binding as B
+    p = B.sar_rda_params_create(B.sar_desc_from_scene(scene, dtype))
+    try:
+        need = B.sar_rda_workspace_bytes(p)
+        assert need == scene.n_azimuth * scene.n_range * (8 if dtype == C64 else 4)
+        ws = torch.zeros(need, dtype=torch.uint8, device="cuda")
+        B.sar_rda_set_workspace(p, ws.data_ptr(), need)
+        rd = to_device_c64(raw)
+        out = torch.zeros_like(rd)
+        st = torch.cuda.current_stream().cuda_stream
+
+        def ws_as_complex():
+            if dtype == C64:
+                return ws.view(torch.complex64).reshape(scene.n_azimuth, scene.n_range).cpu().numpy().astype(np.complex128)
+            return half_to_c128(ws.view(torch.float16).reshape(scene.n_azimuth, scene.n_range, 2))
+
+        if steps:
+            inter = []
+            for s in range(3):
+                B.sar_rda_run_step(rd.data_ptr(), p, out.data_ptr(), s, st)
+                torch.cuda.synchronize()
+                if s < 2:
+                    inter.append(ws_as_complex())
+            return out.cpu().numpy(), inter
+        B.sar_rda_form_image(rd.data_ptr(), p, out.data_ptr(), st)
+        torch.cuda.synchronize()
+        return out.cpu().numpy()
+    finally:
+        B.sar_rda_params_destroy(p)
+
+
+@pytest.fixture(scope="module")
+def small_scene():
+    """1024 pulses x 2048 range samples; a 3 m antenna keeps the aperture (about
+    520 pulses) inside the frame. Same radar otherwise; noise at 20 dB."""
+    sc = inputs.x_band_scene(n_azimuth=1024, n_range=2048, n_targets=0)
+    sc.antenna_m = 3.0
+    sc.targets = inputs.seeded_target_cells(sc, 5, seed=9)
+    raw = inputs.simulate_raw(sc, seed=9)
+    p = oracle.sar_params(sc)
+    rc = oracle.sar_range_compress(p, raw)
+    S = oracle.sar_azimuth_fft(p, rc)
+    img = oracle.sar_azimuth_ifft(p, oracle.sar_azimuth_filter(p, oracle.sar_rcmc(p, S)))
+    return sc, raw, rc, S, img
+
+
+def test_small_scene_each_pass_fp32(small_scene):
+    sc, raw, rc, S, img = small_scene
+    got, inter = _gpu_chain(sc, raw, C64, steps=True)
+    assert rel_l2(inter[0], rc) <= 1e-5                      # fused range compression
+    assert rel_l2(inter[1], S / sc.n_azimuth) <= 1e-5        # azimuth FFT, scaled 1/N_a
+    assert rel_l2(got, img) <= 1e-5
+    for cell in sc.targets:
+        assert quality.peak_cell(got, tuple(cell)) == tuple(cell)
+
+
+def test_small_scene_fp16_intermediates(small_scene):
+    sc, raw, rc, S, img = small_scene
+    got, inter = _gpu_chain(sc, raw, C32H, steps=True)
+    assert rel_l2(inter[0], rc) <= 5e-3
+    assert rel_l2(inter[1], S / sc.n_azimuth) <= 5e-3
+    assert rel_l2(got, img) <= 5e-3
+    for cell in sc.targets:
+        assert quality.peak_cell(got, tuple(cell)) == tuple(cell)
+
+
+def test_single_on_grid_echo_compresses_to_the_pulse_length():
+    sc = inputs.x_band_scene(n_azimuth=1024, n_range=2048, n_targets=0)
+    sc.noise_variance = 0.0
+    raw = np.zeros((1024, 2048), dtype=np.complex64)
+    i = np.arange(-600, 600)
+    kappa = sc.chirp_rate / sc.fs_hz ** 2
+    raw[5, 900 + i] = np.exp(1j * np.pi * kappa * i.astype(np.float64) ** 2)
+    got, inter = _gpu_chain(sc, raw, C64, steps=True)
+    assert abs(inter[0][5, 900] - 1200) < 1e-2
+    assert np.abs(inter[0][6]).max() == 0
+
+
+@pytest.mark.parametrize("dtype,tol", [(C64, 1e-5), (C32H, 5e-3)])
+def test_config4_full_scene(dtype, tol, full_scene):
+    """4096 x 4096, 16 seeded unit targets, noise at 20 dB: whole image and peak cells."""
+    sc, raw, img = full_scene
+    got = _gpu_chain(sc, raw, dtype)
+    err = rel_l2(got, img)
+    assert err <= tol, err
+    for cell in sc.targets:
+        cell = tuple(cell)
+        assert quality.peak_cell(got, cell) == cell
+        assert quality.peak_cell(img, cell) == cell
+    # focus quality matches the reference image's
+    cell = tuple(sc.targets[0])
+    for axis in (0, 1):
+        wg, pg, _ = quality.irw_pslr(quality.cut_through(got.astype(np.complex128), cell, axis))
+        wo, po, _ = quality.irw_pslr(quality.cut_through(img, cell, axis))
+        assert abs(wg - wo) < 0.01 and abs(pg - po) < 0.05
+
+
+@pytest.fixture(scope="module")
+def full_scene():
+    sc = inputs.x_band_scene(n_azimuth=4096, n_range=4096, n_targets=16, seed=4)
+    raw = inputs.simulate_raw(sc, seed=4)
+    img = oracle.sar_rda(oracle.sar_params(sc), raw)
+    return sc, raw, img
