@@ -100,6 +100,29 @@ int fft_plan_destroy(fft_plan_t plan);
  * keys return B200FFT_ERR_INVALID_ARG. Must be called before set_workspace. */
 int fft_plan_set_option(fft_plan_t plan, const char *key, int64_t value);
 
+/* The paper has no counterpart to this call. It is for callers that must not
+ * allocate device memory when they transform: a loop that cannot take the
+ * device-wide stall cudaMalloc or cudaFree may cause, a process whose device
+ * memory is already committed to its own pool, a deployment with a memory
+ * budget fixed at load time. It runs the two-pass transform of `batch`
+ * contiguous complex64 rows of n points (dist = n, in and out DEVICE pointers,
+ * 16-byte aligned, n*batch elements each, in == out allowed) without a plan:
+ * the scratch image and the twiddle tables live in a fixed device array inside
+ * the library (B200FFT_NOALLOC_MAX_ELEMS elements of scratch, 2 MiB, plus
+ * 64 KiB of tables, held by every GPU that loads the library until exit).
+ * Limits: n a power of two, 4096 <= n <= 262144, n*batch <=
+ * B200FFT_NOALLOC_MAX_ELEMS; anything larger returns B200FFT_ERR_WORKSPACE,
+ * other sizes B200FFT_ERR_UNSUPPORTED. It calls no cudaMalloc, cudaFree or
+ * other allocating routine. The first call on a device looks up the array's
+ * device address; make that first call before any stream capture begins.
+ * All calls share the one array: two calls that overlap on the GPU (different
+ * streams, no ordering between them) race on it, so order them. The array keeps
+ * the previous call's contents; each call rebuilds the tables it needs and
+ * overwrites the scratch it reads, so no clearing is required of the caller.
+ * Results equal those of a four-step plan of the same size. */
+#define B200FFT_NOALLOC_MAX_ELEMS 262144
+int fft_execute_noalloc(int64_t n, int64_t batch, int direction, const void *in, void *out, void *stream);
+
 /* Static description of a status code. */
 const char *fft_status_string(int status);
 

@@ -24,7 +24,7 @@ EXPORTS = [
     "fft_execute_host", "fft_plan_destroy", "fft_plan_set_option", "fft_status_string",
     "b200fft_launch_count", "sar_rda_params_create", "sar_rda_workspace_bytes",
     "sar_rda_set_workspace", "sar_rda_form_image", "sar_rda_form_image_host", "sar_rda_run_step",
-    "sar_rda_params_destroy",
+    "sar_rda_params_destroy", "fft_execute_noalloc",
 ]
 
 
@@ -68,6 +68,7 @@ def _load():
     L.sar_rda_form_image_host.argtypes = [vp, vp, vp, vp, vp, vp]
     L.sar_rda_run_step.argtypes = [vp, vp, vp, ci, vp]
     L.sar_rda_params_destroy.argtypes = [vp]
+    L.fft_execute_noalloc.argtypes = [i64, i64, ci, vp, vp, vp]
     return L
 
 
@@ -117,6 +118,17 @@ def fft_execute(plan, in_ptr, out_ptr, stream=0):
 
 def fft_execute_host(plan, host_in, host_out, dev_in, dev_out, stream=0):
     _check(_lib.fft_execute_host(plan, host_in, host_out, dev_in, dev_out, stream), "fft_execute_host")
+
+
+def fft_execute_noalloc(n, batch, direction, in_ptr, out_ptr, stream=0):
+    """Two-pass transform of `batch` contiguous complex64 rows of n points that
+    allocates nothing: scratch and tables live in a fixed array inside the
+    library (n * batch <= NOALLOC_MAX_ELEMS). For callers that cannot call
+    cudaMalloc while they process. Calls sharing the GPU must be ordered."""
+    _check(_lib.fft_execute_noalloc(n, batch, direction, in_ptr, out_ptr, stream), "fft_execute_noalloc")
+
+
+NOALLOC_MAX_ELEMS = 262144
 
 
 def fft_plan_destroy(plan):

@@ -191,6 +191,55 @@ int fourstep_build(FourStep* fs, int64_t n, int64_t batch, int64_t dist, int dir
     return B200FFT_OK;
 }
 
+static int fourstep_split(int64_t n, int64_t* n1, int64_t* n2) {
+    int lg = 0;
+    while (((int64_t)1 << lg) < n) ++lg;
+    if (((int64_t)1 << lg) != n || lg < 12 || lg > 20) return B200FFT_ERR_UNSUPPORTED;
+    *n1 = (int64_t)1 << ((lg + 1) / 2);
+    *n2 = n / *n1;
+    return B200FFT_OK;
+}
+
+size_t fourstep_table_elems(int64_t n, int direction, int dtype) {
+    int64_t n1, n2;
+    if (fourstep_split(n, &n1, &n2) != B200FFT_OK) return 0;
+    const bool inv = direction == B200FFT_INVERSE;
+    const FourStepEntry* p1 = find(k_pass1, (int)n1, inv, dtype);
+    const FourStepEntry* p2 = find(k_pass2, (int)n2, inv, dtype);
+    if (!p1 || !p2) return 0;
+    // each table starts on a 16-byte boundary (two float2)
+    auto up = [](size_t v) { return (v + 1) & ~(size_t)1; };
+    return up((size_t)p1->tw_total) + up((size_t)p2->tw_total) + 1024 + up((size_t)(n / 1024));
+}
+
+int fourstep_build_in_place(FourStep* fs, int64_t n, int64_t batch, int64_t dist, int direction, int dtype,
+                            float2* tables, size_t table_elems, cudaStream_t st) {
+    *fs = FourStep();
+    int64_t n1, n2;
+    int rc = fourstep_split(n, &n1, &n2);
+    if (rc != B200FFT_OK) return rc;
+    const size_t need = fourstep_table_elems(n, direction, dtype);
+    if (need == 0) return B200FFT_ERR_UNSUPPORTED;
+    if (!tables || table_elems < need) return B200FFT_ERR_WORKSPACE;
+    const bool inv = direction == B200FFT_INVERSE;
+    fs->n = n; fs->n1 = n1; fs->n2 = n2; fs->batch = batch; fs->dist = dist;
+    fs->direction = direction; fs->dtype = dtype;
+    fs->pass1 = find(k_pass1, (int)n1, inv, dtype);
+    fs->pass2 = find(k_pass2, (int)n2, inv, dtype);
+    auto up = [](size_t v) { return (v + 1) & ~(size_t)1; };
+    const int hi_count = (int)(n / 1024);
+    fs->tw1 = tables;
+    fs->tw2 = fs->tw1 + up((size_t)fs->pass1->tw_total);
+    fs->tw_lo = fs->tw2 + up((size_t)fs->pass2->tw_total);
+    fs->tw_hi = fs->tw_lo + 1024;
+    bool ok = fs->pass1->build_tw(fs->tw1, st) == cudaSuccess && fs->pass2->build_tw(fs->tw2, st) == cudaSuccess;
+    build_factor_table<<<4, 256, 0, st>>>(fs->tw_lo, 1024, 1, n);
+    build_factor_table<<<(hi_count + 255) / 256, 256, 0, st>>>(fs->tw_hi, hi_count, 1024, n);
+    g_launch_count.fetch_add(2, std::memory_order_relaxed);
+    ok = ok && cudaGetLastError() == cudaSuccess;
+    return ok ? B200FFT_OK : B200FFT_ERR_CUDA;
+}
+
 int fourstep_execute(const FourStep* fs, const void* in, void* out, void* workspace, cudaStream_t st) {
     FourStepArgs a;
     a.tw_lo = fs->tw_lo;

@@ -22,4 +22,13 @@ int fourstep_build(FourStep* fs, int64_t n, int64_t batch, int64_t dist, int dir
 int fourstep_execute(const FourStep* fs, const void* in, void* out, void* workspace, cudaStream_t st);
 void fourstep_release(FourStep* fs);
 
+// Number of float2 table entries a FourStep of this size needs (0 if unsupported).
+size_t fourstep_table_elems(int64_t n, int direction, int dtype);
+// Like fourstep_build, but allocates nothing: the four tables are placed in
+// caller-provided device memory `tables` (at least fourstep_table_elems entries)
+// and built by kernels enqueued on `st`, without synchronising. The FourStep
+// must not be passed to fourstep_release.
+int fourstep_build_in_place(FourStep* fs, int64_t n, int64_t batch, int64_t dist, int direction, int dtype,
+                            float2* tables, size_t table_elems, cudaStream_t st);
+
 }  // namespace b200fft
