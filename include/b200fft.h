@@ -96,8 +96,12 @@ int fft_plan_destroy(fft_plan_t plan);
 
 /* Test knob: force a kernel variant (paper, Section "One Pass": "a regression
  * test forces N=8192 through this path"). key "four_step" value 1 routes a
- * rows plan of any supported n >= 4096 through the two-pass split. Unknown
- * keys return B200FFT_ERR_INVALID_ARG. Must be called before set_workspace. */
+ * rows plan of any supported n >= 4096 through the two-pass split. Key
+ * "cluster" value c (1, 2 or 4; 0 = the default for that size) picks the
+ * variant of a single-pass plan in which c CTAs of one thread-block cluster
+ * share a tile through distributed shared memory; B200FFT_ERR_UNSUPPORTED if
+ * that variant is not compiled for the plan's size. Unknown keys return
+ * B200FFT_ERR_INVALID_ARG. Must be called before set_workspace. */
 int fft_plan_set_option(fft_plan_t plan, const char *key, int64_t value);
 
 /* The paper has no counterpart to this call. It is for callers that must not

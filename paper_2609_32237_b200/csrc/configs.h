@@ -1,27 +1,37 @@
-// Radix factorisations of the compiled sizes. Cfg<N, W, P, G, r1, r2, r3, r4>:
-// N points, W transforms per tile, P values per thread, G tiles per CTA.
+// Radix factorisations of the compiled sizes. Cfg<N, W, P, G, CL, r1, r2, r3, r4>:
+// N points, W transforms per tile, P values per thread, G tiles per CTA, CL CTAs
+// (one thread-block cluster) sharing a tile through distributed shared memory.
 #pragma once
 #include "fft_core.cuh"
 
 namespace b200fft {
 
 // contiguous rows, one transform per tile
-using R256 = Cfg<256, 1, 32, 16, 16, 16>;
-using R512 = Cfg<512, 1, 32, 8, 16, 2, 16>;
-using R1024 = Cfg<1024, 1, 32, 4, 16, 4, 16>;
-using R2048 = Cfg<2048, 1, 32, 2, 16, 8, 16>;
-using R4096 = Cfg<4096, 1, 32, 1, 16, 16, 16>;
-using R8192 = Cfg<8192, 1, 32, 1, 16, 32, 16>;
-using R16384 = Cfg<16384, 1, 32, 1, 16, 4, 16, 16>;
+using R256 = Cfg<256, 1, 32, 16, 1, 16, 16>;
+using R512 = Cfg<512, 1, 32, 8, 1, 16, 2, 16>;
+using R1024 = Cfg<1024, 1, 32, 4, 1, 16, 4, 16>;
+using R2048 = Cfg<2048, 1, 32, 2, 1, 16, 8, 16>;
+using R4096 = Cfg<4096, 1, 32, 1, 1, 16, 16, 16>;
+using R8192 = Cfg<8192, 1, 32, 1, 1, 16, 32, 16>;
+using R16384 = Cfg<16384, 1, 32, 1, 1, 16, 4, 16, 16>;
+// the same transforms split over a cluster of 2 or 4 CTAs (smaller tiles per SM, more CTAs resident)
+using R8192x2 = Cfg<8192, 1, 32, 1, 2, 16, 32, 16>;
+using R8192x4 = Cfg<8192, 1, 32, 1, 4, 16, 32, 16>;
+using R16384x2 = Cfg<16384, 1, 32, 1, 2, 16, 4, 16, 16>;
+using R16384x4 = Cfg<16384, 1, 32, 1, 4, 16, 4, 16, 16>;
 
 // W adjacent columns (or rows, in the second pass of the two-pass split) per tile
-using T64 = Cfg<64, 4, 32, 16, 16, 4>;
-using T128 = Cfg<128, 4, 32, 8, 16, 8>;
-using T256 = Cfg<256, 4, 32, 4, 16, 16>;
-using T512 = Cfg<512, 4, 32, 2, 16, 2, 16>;
-using T1024 = Cfg<1024, 4, 32, 1, 16, 4, 16>;
-using T2048 = Cfg<2048, 4, 32, 1, 16, 8, 16>;
-using T4096 = Cfg<4096, 4, 32, 1, 16, 16, 16>;
-using T8192 = Cfg<8192, 2, 32, 1, 16, 32, 16>;
+using T64 = Cfg<64, 4, 32, 16, 1, 16, 4>;
+using T128 = Cfg<128, 4, 32, 8, 1, 16, 8>;
+using T256 = Cfg<256, 4, 32, 4, 1, 16, 16>;
+using T512 = Cfg<512, 4, 32, 2, 1, 16, 2, 16>;
+using T1024 = Cfg<1024, 4, 32, 1, 1, 16, 4, 16>;
+using T2048 = Cfg<2048, 4, 32, 1, 1, 16, 8, 16>;
+using T4096 = Cfg<4096, 4, 32, 1, 1, 16, 16, 16>;
+using T8192 = Cfg<8192, 2, 32, 1, 1, 16, 32, 16>;
+using T2048x2 = Cfg<2048, 4, 32, 1, 2, 16, 8, 16>;
+using T4096x2 = Cfg<4096, 4, 32, 1, 2, 16, 16, 16>;
+using T4096x4 = Cfg<4096, 4, 32, 1, 4, 16, 16, 16>;
+using T8192x2 = Cfg<8192, 2, 32, 1, 2, 16, 32, 16>;
 
 }  // namespace b200fft

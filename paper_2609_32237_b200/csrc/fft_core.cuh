@@ -161,9 +161,9 @@ struct Dft<32> {
 };
 
 // ------------------------------------------------------------ configuration
-template <int N_, int W_, int P_, int G_, int R1_, int R2_, int R3_ = 1, int R4_ = 1>
+template <int N_, int W_, int P_, int G_, int CL_, int R1_, int R2_, int R3_ = 1, int R4_ = 1>
 struct Cfg {
-    static constexpr int N = N_, W = W_, P = P_, G = G_;
+    static constexpr int N = N_, W = W_, P = P_, G = G_, CL = CL_;
     static constexpr int S = (R3_ == 1) ? 2 : ((R4_ == 1) ? 3 : 4);
     __host__ __device__ static constexpr int radix(int s) { return s == 1 ? R1_ : (s == 2 ? R2_ : (s == 3 ? R3_ : R4_)); }
     __host__ __device__ static constexpr int L(int s) {
@@ -171,10 +171,14 @@ struct Cfg {
         for (int i = 1; i <= s; ++i) l /= radix(i);
         return l;
     }
-    static constexpr int T = N * W / P;       // threads per tile
+    // A tile (W transforms of N points) is shared by a cluster of CL CTAs: each keeps
+    // 1/CL of it in its own shared memory and 1/CL of the threads.
+    static constexpr int T = N * W / P / CL;  // threads per tile per CTA
     static constexpr int THREADS = T * G;     // threads per CTA
     static constexpr int TILE_ELEMS = N * W;
-    static constexpr int SMEM_BYTES = TILE_ELEMS * G * 8;
+    static constexpr int LOCAL_ELEMS = TILE_ELEMS / CL;
+    static constexpr int SMEM_BYTES = LOCAL_ELEMS * G * 8;
+    static constexpr int RC = R1_ / CL;       // values of the top digit a CTA owns after the first exchange
     // twiddle rows of stage s < S start here: (radix-1) rows of L(s) entries each
     __host__ __device__ static constexpr int tw_off(int s) {
         int o = 0;
@@ -182,56 +186,126 @@ struct Cfg {
         return o;
     }
     static constexpr int TW_TOTAL = tw_off(S);
+    // Index, within the whole tile, of butterfly v (0 .. V-1) of thread t of CTA `rank`
+    // at a stage with V butterflies per thread. Butterflies go to threads in adjacent
+    // pairs, and the pairs of one register slot are contiguous across the threads of a
+    // CTA, so that a warp's shared-memory access is one contiguous run.
+    template <int V>
+    __host__ __device__ static constexpr int cidx(int t, int v, int rank) {
+        if (V == 1) return rank * T + t;
+        return rank * V * T + 2 * ((v >> 1) * T + t) + (v & 1);
+    }
+    // weight of digit i (1 .. S-1) in the last stage's local butterfly index (top digit fastest)
+    __host__ __device__ static constexpr int blw(int i) {
+        int w = 1;
+        if (i >= 2) w = RC;
+        for (int k = 2; k < i; ++k) w *= radix(k);
+        return w;
+    }
     static_assert(R1_ * R2_ * R3_ * R4_ == N_, "radices must multiply to N");
     static_assert(L(1) * W_ >= 16, "the swizzle permutes 16-element groups below the top digit");
+    static_assert(CL_ == 1 || G_ == 1, "a cluster works on one tile");
+    static_assert(CL_ >= 1 && R1_ % CL_ == 0 && RC >= 2, "the cluster splits the top digit");
+    static_assert(CL_ == 1 || RC * W_ >= 16 || L(2) * W_ >= 16, "second digit must stay constant over 16 elements");
     // registers per thread are capped at 128 so that at least 65536 / (128 * THREADS) CTAs fit an SM
     static constexpr int MINB = (65536 / (128 * THREADS)) > 0 ? (65536 / (128 * THREADS)) : 1;
     static_assert(P_ % R1_ == 0 && P_ % R2_ == 0 && P_ % R3_ == 0 && P_ % R4_ == 0, "P must be a multiple of every radix");
     static_assert(P_ / R1_ >= 2 && P_ / radix(S) >= 2, "first and last stage need two butterflies per thread for 128-bit access");
-    static_assert((N_ * W_) % P_ == 0, "tile must divide among threads");
+    static_assert((N_ * W_) % (P_ * CL_) == 0, "tile must divide among threads");
 };
 
-// Geometry of butterfly v of thread t at stage s.
+// Geometry of butterfly v of thread te (index within the whole tile: cluster rank * T + t)
+// at stage s. Element indices are local to the owning CTA's shared memory.
 template <class C, int s>
 struct Geo {
     static constexpr int r = C::radix(s), V = C::P / r, Ls = C::L(s), Lp = C::L(s - 1), L1 = C::L(1);
     static constexpr bool last = (s == C::S);
-    static constexpr int W = C::W;
+    static constexpr int W = C::W, CL = C::CL, RC = C::RC;
     static constexpr int estep = last ? W : Ls * W;  // element step per register index j
-    int e0;    // element index (position * W + column) of j = 0, before swizzle
-    int mask;  // swizzle for s > 1
-    int lo;    // twiddle column (stages < S); output index low part (last stage)
+    int e0;    // local element index (position * W + column) of j = 0, before swizzle
+    int bl0;   // low bits of the last-stage butterfly index of these positions, digit s counted as 0
+    int lo;    // twiddle column (stages < S); global output index low part (last stage)
 
-    __device__ __forceinline__ void init(int t, int v) {
-        const int c = V * t + v;
+    // low 4 bits of the last stage's local butterfly index that position p0 belongs to,
+    // leaving out digit `skip`; the top digit is taken relative to the owning CTA
+    template <int skip>
+    static __device__ __forceinline__ int bl_of(int p0, int rank) {
+        int bl = 0;
+        static_for<1, C::S>([&](auto i_) {
+            constexpr int i = decltype(i_)::value;
+            if constexpr (i != skip && C::blw(i) < 16) {
+                int d = (p0 / C::L(i)) % C::radix(i);
+                if constexpr (i == 1) d -= rank * RC;
+                bl += d * C::blw(i);
+            }
+        });
+        return bl;
+    }
+
+    __device__ __forceinline__ void init(int t, int v, int rank) {
+        const int c = C::template cidx<V>(t, v, rank);
         const int q = c % W;
         const int b = c / W;
         if constexpr (!last) {
             lo = b % Ls;
             const int hi = b / Ls;
-            const int p0 = hi * Lp + lo;
-            e0 = p0 * W + q;
-            mask = ((p0 / L1) * W) & 14;
+            const int p0 = hi * Lp + lo;              // position with digit s = 0
+            bl0 = bl_of<s>(p0, rank);
+            e0 = p0 * W + q - ((s == 1) ? 0 : rank * C::LOCAL_ELEMS);
         } else {
-            int rem = b, p0 = 0, d1 = 0;
-            static_for<1, C::S>([&](auto i_) {
+            const int bloc = b - rank * (C::N / r / CL);   // local butterfly index, top digit fastest
+            const int d1 = bloc % RC + rank * RC;
+            int rem = bloc / RC, p0 = d1 * L1;
+            lo = d1 + C::radix(1) * rem;
+            static_for<2, C::S>([&](auto i_) {
                 constexpr int i = decltype(i_)::value;
-                const int d = rem % C::radix(i);
+                p0 += (rem % C::radix(i)) * C::L(i);
                 rem /= C::radix(i);
-                p0 += d * C::L(i);
-                if constexpr (i == 1) d1 = d;
             });
-            e0 = p0 * W + q;
-            mask = (d1 * W) & 14;
-            lo = b;
+            e0 = p0 * W + q - rank * C::LOCAL_ELEMS;
+            bl0 = bloc & 15;
         }
     }
+    // CTA (cluster rank) that owns position j of the first stage after the first exchange
+    template <int j>
+    __host__ __device__ static constexpr int dest() { return j / RC; }
     template <int j>
     __device__ __forceinline__ int elem() const {
-        if constexpr (s == 1) return (e0 + j * estep) ^ ((j * W) & 14);
-        else return (e0 + j * estep) ^ mask;
+        if constexpr (s == 1) {
+            constexpr int jl = j % RC;                // top digit relative to the owner
+            return (e0 + jl * estep) ^ (((bl0 + jl) * W) & 14);
+        } else if constexpr (!last) {
+            if constexpr (C::blw(s) < 16) return (e0 + j * estep) ^ (((bl0 + j * C::blw(s)) * W) & 14);
+            else return (e0 + j * estep) ^ ((bl0 * W) & 14);
+        } else {
+            return (e0 + j * estep) ^ ((bl0 * W) & 14);
+        }
     }
 };
+
+// ------------------------------------------------------------ cluster helpers
+__device__ __forceinline__ unsigned cluster_ctarank() {
+    unsigned r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory"); }
+__device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
+// store two complex values into the shared memory of CTA `rank` of this cluster, at the
+// address that `local` has in this CTA (all CTAs of a cluster lay out shared memory alike)
+__device__ __forceinline__ void st_cluster_f4(const float2* local, unsigned rank, float4 v) {
+    const unsigned a = (unsigned)__cvta_generic_to_shared(local);
+    unsigned ra;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(ra) : "r"(a), "r"(rank));
+    asm volatile("st.shared::cluster.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(ra), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w)
+                 : "memory");
+}
+__device__ __forceinline__ void st_cluster_f2(const float2* local, unsigned rank, float2 v) {
+    const unsigned a = (unsigned)__cvta_generic_to_shared(local);
+    unsigned ra;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(ra) : "r"(a), "r"(rank));
+    asm volatile("st.shared::cluster.v2.f32 [%0], {%1, %2};" ::"r"(ra), "f"(v.x), "f"(v.y) : "memory");
+}
 
 // ------------------------------------------------------------ storage types
 struct StoreC64 {
@@ -271,21 +345,32 @@ struct StoreC32H {
 // ------------------------------------------------------------ the engine
 template <class C>
 struct Engine {
-    static constexpr int P = C::P, W = C::W, S = C::S;
+    static constexpr int P = C::P, W = C::W, S = C::S, CL = C::CL;
     float2 x[P];
+    int rank;   // CTA rank in its cluster (0 when CL == 1)
+    int t;      // thread index within the tile's threads of this CTA
+
+    __device__ __forceinline__ void setup(int t_) {
+        rank = (CL > 1) ? (int)cluster_ctarank() : 0;
+        t = t_;
+        // every CTA of the cluster must be running before its shared memory is written remotely
+        if constexpr (CL > 1) cluster_arrive();
+    }
 
     // ---- shared-memory exchange -------------------------------------------------
     // Registers of stage s are x[j * V + v]: butterfly v, element j.
     template <int s, bool WR>
-    __device__ __forceinline__ void smem_rw(float2* sm, int t) {
+    __device__ __forceinline__ void smem_rw(float2* sm) {
         using G = Geo<C, s>;
         constexpr int V = G::V, r = G::r;
+        constexpr bool REMOTE = (CL > 1 && s == 1);
+        static_assert(!(REMOTE && !WR), "with a cluster the first stage reads global memory only");
         if constexpr (G::last && W == 1) {
             // the two butterflies of a thread sit L1 apart: go 128-bit along j instead
             static_for<0, V>([&](auto v_) {
                 constexpr int v = decltype(v_)::value;
                 G g;
-                g.init(t, v);
+                g.init(t, v, rank);
                 static_for<0, r / 2>([&](auto h_) {
                     constexpr int j = 2 * decltype(h_)::value;
                     float4* p = reinterpret_cast<float4*>(sm + g.template elem<j>());
@@ -302,14 +387,16 @@ struct Engine {
             static_for<0, V / 2>([&](auto h_) {
                 constexpr int v = 2 * decltype(h_)::value;
                 G g;
-                g.init(t, v);
+                g.init(t, v, rank);
                 static_for<0, r>([&](auto j_) {
                     constexpr int j = decltype(j_)::value;
-                    float4* p = reinterpret_cast<float4*>(sm + g.template elem<j>());
+                    float2* p2 = sm + g.template elem<j>();
                     if constexpr (WR) {
-                        *p = make_float4(x[j * V + v].x, x[j * V + v].y, x[j * V + v + 1].x, x[j * V + v + 1].y);
+                        const float4 val = make_float4(x[j * V + v].x, x[j * V + v].y, x[j * V + v + 1].x, x[j * V + v + 1].y);
+                        if constexpr (REMOTE) st_cluster_f4(p2, (unsigned)G::template dest<j>(), val);
+                        else *reinterpret_cast<float4*>(p2) = val;
                     } else {
-                        const float4 q = *p;
+                        const float4 q = *reinterpret_cast<const float4*>(p2);
                         x[j * V + v] = make_float2(q.x, q.y);
                         x[j * V + v + 1] = make_float2(q.z, q.w);
                     }
@@ -317,12 +404,28 @@ struct Engine {
             });
         } else {
             G g;
-            g.init(t, 0);
+            g.init(t, 0, rank);
             static_for<0, r>([&](auto j_) {
                 constexpr int j = decltype(j_)::value;
-                if constexpr (WR) sm[g.template elem<j>()] = x[j];
-                else x[j] = sm[g.template elem<j>()];
+                float2* p2 = sm + g.template elem<j>();
+                if constexpr (WR) {
+                    if constexpr (REMOTE) st_cluster_f2(p2, (unsigned)G::template dest<j>(), x[j]);
+                    else *p2 = x[j];
+                } else {
+                    x[j] = *p2;
+                }
             });
+        }
+    }
+
+    // barrier of exchange s -> s+1 (DIF) or s -> s-1 (DIT)
+    template <bool CLUSTER>
+    __device__ __forceinline__ void exchange_barrier() {
+        if constexpr (CLUSTER) {
+            cluster_arrive();
+            cluster_wait();
+        } else {
+            __syncthreads();
         }
     }
 
@@ -330,7 +433,7 @@ struct Engine {
     // DIT = false: butterfly, then multiply output k by tw[k][lo]   (stages 1..S-1)
     // DIT = true : multiply input j by tw[j][lo], then butterfly     (transposed network)
     template <int s, bool DIT>
-    __device__ __forceinline__ void compute(const float2* __restrict__ tw, int t) {
+    __device__ __forceinline__ void compute(const float2* __restrict__ tw) {
         using G = Geo<C, s>;
         constexpr int V = G::V, r = G::r, Ls = G::Ls;
         constexpr bool has_tw = !G::last;
@@ -361,9 +464,7 @@ struct Engine {
                 });
                 [[maybe_unused]] int lo0 = 0;
                 if constexpr (has_tw) {
-                    G g;
-                    g.init(t, v);
-                    lo0 = g.lo;
+                    lo0 = (C::template cidx<V>(t, v, rank) / W) % Ls;
                     if constexpr (DIT) twiddle_pair(lo0, a, b);
                 }
                 Dft<r>::run(a);
@@ -378,9 +479,7 @@ struct Engine {
         } else {
             [[maybe_unused]] int lo0 = 0;
             if constexpr (has_tw) {
-                G g;
-                g.init(t, 0);
-                lo0 = g.lo;
+                lo0 = (C::template cidx<1>(t, 0, rank) / W) % Ls;
                 if constexpr (DIT) twiddle_pair(lo0, x, nullptr);
             }
             Dft<r>::run(x);
@@ -392,12 +491,12 @@ struct Engine {
     // position of register (j, v): p = j * L1 + lo; rows: index base + p (+1 for v odd);
     // columns: index base + p * ld + q.
     template <class ST, bool CONJ>
-    __device__ __forceinline__ void load_first(const void* in, int64_t base, int64_t ld, int t) {
+    __device__ __forceinline__ void load_first(const void* in, int64_t base, int64_t ld) {
         using G = Geo<C, 1>;
         constexpr int V = G::V, r = G::r;
         static_for<0, V / 2>([&](auto h_) {
             constexpr int v = 2 * decltype(h_)::value;
-            const int c = V * t + v;
+            const int c = C::template cidx<V>(t, v, rank);
             const int q = c % W, lo = c / W;
             static_for<0, r>([&](auto j_) {
                 constexpr int j = decltype(j_)::value;
@@ -411,12 +510,12 @@ struct Engine {
         });
     }
     template <class ST, bool CONJ>
-    __device__ __forceinline__ void store_first(void* out, int64_t base, int64_t ld, int t, float scale) {
+    __device__ __forceinline__ void store_first(void* out, int64_t base, int64_t ld, float scale) {
         using G = Geo<C, 1>;
         constexpr int V = G::V, r = G::r;
         static_for<0, V / 2>([&](auto h_) {
             constexpr int v = 2 * decltype(h_)::value;
-            const int c = V * t + v;
+            const int c = C::template cidx<V>(t, v, rank);
             const int q = c % W, lo = c / W;
             static_for<0, r>([&](auto j_) {
                 constexpr int j = decltype(j_)::value;
@@ -428,16 +527,23 @@ struct Engine {
             });
         });
     }
-    // ---- global store with the last-stage mapping: X[lo + (N / r_S) j] ---------------------
+    // output index (low part) and column of butterfly pair v of the last stage
+    __device__ __forceinline__ void last_index(int v, int& b0, int& q) const {
+        Geo<C, S> g;
+        g.init(t, v, rank);
+        b0 = g.lo;
+        q = C::template cidx<Geo<C, S>::V>(t, v, rank) % W;
+    }
+    // ---- global store with the last-stage mapping: X[b0 + (N / r_S) j] ---------------------
     template <class ST, bool CONJ>
-    __device__ __forceinline__ void store_last(void* out, int64_t base, int64_t ld, int t, float scale) {
+    __device__ __forceinline__ void store_last(void* out, int64_t base, int64_t ld, float scale) {
         using G = Geo<C, S>;
         constexpr int V = G::V, r = G::r;
         constexpr int KS = C::N / r;
         static_for<0, V / 2>([&](auto h_) {
             constexpr int v = 2 * decltype(h_)::value;
-            const int c = V * t + v;
-            const int q = c % W, b0 = c / W;
+            int b0, q;
+            last_index(v, b0, q);
             static_for<0, r>([&](auto j_) {
                 constexpr int j = decltype(j_)::value;
                 const int64_t idx = (W == 1) ? base + j * KS + b0 : base + (int64_t)(j * KS + b0) * ld + q;
@@ -451,28 +557,30 @@ struct Engine {
 
     // ---- whole networks ---------------------------------------------------------------
     // registers hold stage-1 layout on entry; on exit they hold the last stage's
-    // layout: x[j*V + v] = X[b' + (N/r_S) j] for butterfly b' (digit-reversed positions)
-    __device__ __forceinline__ void dif(float2* sm, const float2* __restrict__ tw, int t) {
+    // layout: x[j*V + v] = X[b0 + (N/r_S) j] for butterfly pair v (digit-reversed positions)
+    __device__ __forceinline__ void dif(float2* sm, const float2* __restrict__ tw) {
         static_for<1, S + 1>([&](auto s_) {
             constexpr int s = decltype(s_)::value;
-            compute<s, false>(tw, t);
+            compute<s, false>(tw);
             if constexpr (s < S) {
-                smem_rw<s, true>(sm, t);
-                __syncthreads();
-                smem_rw<s + 1, false>(sm, t);
+                if constexpr (CL > 1 && s == 1) cluster_wait();   // pairs with the arrive in setup()
+                smem_rw<s, true>(sm);
+                exchange_barrier<(CL > 1 && s == 1)>();
+                smem_rw<s + 1, false>(sm);
             }
         });
     }
     // registers hold the last stage's layout (digit-reversed positions) on entry,
     // stage-1 layout in natural order on exit
-    __device__ __forceinline__ void dit(float2* sm, const float2* __restrict__ tw, int t) {
+    __device__ __forceinline__ void dit(float2* sm, const float2* __restrict__ tw) {
+        static_assert(CL == 1, "the backward network is built for single-CTA tiles");
         static_for<0, S>([&](auto i_) {
             constexpr int s = S - decltype(i_)::value;
-            compute<s, true>(tw, t);
+            compute<s, true>(tw);
             if constexpr (s > 1) {
-                smem_rw<s, true>(sm, t);
+                smem_rw<s, true>(sm);
                 __syncthreads();
-                smem_rw<s - 1, false>(sm, t);
+                smem_rw<s - 1, false>(sm);
             }
         });
     }
@@ -487,20 +595,22 @@ struct FftArgs {
     float scale;
 };
 
-// One CTA = G tiles. INV: inverse via conj(FFT(conj(x))) * scale.
+// One CTA = G tiles, or one cluster of CL CTAs = one tile. INV: inverse via
+// conj(FFT(conj(x))) * scale.
 template <class C, bool INV, class TIn, class TOut>
 __global__ void __launch_bounds__(C::THREADS, C::MINB) fft_kernel(const FftArgs a) {
     extern __shared__ __align__(16) float2 smem_dyn[];
     const int g = threadIdx.x / C::T, t = threadIdx.x % C::T;
-    int64_t tile = (int64_t)blockIdx.x * C::G + g;
+    int64_t tile = (C::CL > 1) ? (int64_t)(blockIdx.x / C::CL) : (int64_t)blockIdx.x * C::G + g;
     const bool active = tile < a.tiles;
     if (!active) tile = a.tiles - 1;          // keep the barriers uniform; results discarded
-    float2* sm = smem_dyn + g * C::TILE_ELEMS;
+    float2* sm = smem_dyn + g * C::LOCAL_ELEMS;
     const int64_t base = (C::W == 1) ? tile * a.dist : tile * C::W;
     Engine<C> e;
-    e.template load_first<TIn, INV>(a.in, base, a.dist, t);
-    e.dif(sm, a.tw, t);
-    if (active) e.template store_last<TOut, INV>(a.out, base, a.dist, t, a.scale);
+    e.setup(t);
+    e.template load_first<TIn, INV>(a.in, base, a.dist);
+    e.dif(sm, a.tw);
+    if (active) e.template store_last<TOut, INV>(a.out, base, a.dist, a.scale);
 }
 
 // Builds the per-stage twiddle rows of a configuration in float64, rounds once to fp32:

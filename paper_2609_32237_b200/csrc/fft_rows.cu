@@ -8,11 +8,16 @@ static const KernelEntry k_rows[] = {
     B200FFT_ENTRIES_STD(R256),  B200FFT_ENTRIES_STD(R512),
     B200FFT_ENTRIES_STD(R1024), B200FFT_ENTRIES_STD(R2048), B200FFT_ENTRIES_STD(R4096),
     B200FFT_ENTRIES_STD(R8192), B200FFT_ENTRIES_STD(R16384),
+    B200FFT_ENTRIES_STD(R8192x2), B200FFT_ENTRIES_STD(R8192x4),
+    B200FFT_ENTRIES_STD(R16384x2), B200FFT_ENTRIES_STD(R16384x4),
 };
 
-const KernelEntry* find_rows_kernel(int n, bool inverse, int in_dtype, int out_dtype) {
+static int default_cluster(int n) { return 1; }
+
+const KernelEntry* find_rows_kernel(int n, bool inverse, int in_dtype, int out_dtype, int cl) {
+    if (cl == 0) cl = default_cluster(n);
     for (const KernelEntry& e : k_rows)
-        if (e.n == n && e.inverse == inverse && e.in_dtype == in_dtype && e.out_dtype == out_dtype) return &e;
+        if (e.n == n && e.cl == cl && e.inverse == inverse && e.in_dtype == in_dtype && e.out_dtype == out_dtype) return &e;
     return nullptr;
 }
 

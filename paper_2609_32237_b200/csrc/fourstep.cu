@@ -44,22 +44,23 @@ __global__ void __launch_bounds__(C::THREADS, C::MINB) fourstep_pass1_kernel(con
     extern __shared__ __align__(16) float2 smem_dyn[];
     constexpr int W = C::W;
     const int g = threadIdx.x / C::T, t = threadIdx.x % C::T;
-    int64_t tile = (int64_t)blockIdx.x * C::G + g;
+    int64_t tile = (C::CL > 1) ? (int64_t)(blockIdx.x / C::CL) : (int64_t)blockIdx.x * C::G + g;
     const bool active = tile < a.tiles;
     if (!active) tile = a.tiles - 1;
     const int64_t b = tile / a.groups, cg = tile % a.groups;
-    float2* sm = smem_dyn + g * C::TILE_ELEMS;
+    float2* sm = smem_dyn + g * C::LOCAL_ELEMS;
     Engine<C> e;
-    e.template load_first<TIn, INV>(a.in, b * a.dist_in + cg * W, a.n2, t);
-    e.dif(sm, a.tw, t);
+    e.setup(t);
+    e.template load_first<TIn, INV>(a.in, b * a.dist_in + cg * W, a.n2);
+    e.dif(sm, a.tw);
     if (!active) return;
     using G = Geo<C, C::S>;
     constexpr int V = G::V, r = G::r, KS = C::N / r;
     const int64_t nmask = a.n - 1;
     static_for<0, V / 2>([&](auto h_) {
         constexpr int v = 2 * decltype(h_)::value;
-        const int c = V * t + v;
-        const int q = c % W, b0 = c / W;
+        int b0, q;
+        e.last_index(v, b0, q);
         const int64_t j2 = cg * W + q;
         static_for<0, r>([&](auto j_) {
             constexpr int j = decltype(j_)::value;
@@ -77,19 +78,20 @@ __global__ void __launch_bounds__(C::THREADS, C::MINB) fourstep_pass2_kernel(con
     extern __shared__ __align__(16) float2 smem_dyn[];
     constexpr int W = C::W;
     const int g = threadIdx.x / C::T, t = threadIdx.x % C::T;
-    int64_t tile = (int64_t)blockIdx.x * C::G + g;
+    int64_t tile = (C::CL > 1) ? (int64_t)(blockIdx.x / C::CL) : (int64_t)blockIdx.x * C::G + g;
     const bool active = tile < a.tiles;
     if (!active) tile = a.tiles - 1;
     const int64_t b = tile / a.groups, rg = tile % a.groups;
-    float2* sm = smem_dyn + g * C::TILE_ELEMS;
+    float2* sm = smem_dyn + g * C::LOCAL_ELEMS;
     Engine<C> e;
+    e.setup(t);
     {
         using G = Geo<C, 1>;
         constexpr int V = G::V, r = G::r;
         const int64_t rowbase = b * a.dist_in + rg * W * a.n2;
         static_for<0, V / 2>([&](auto h_) {
             constexpr int v = 2 * decltype(h_)::value;
-            const int c = V * t + v;
+            const int c = C::template cidx<V>(e.t, v, e.rank);
             const int q = c % W, lo = c / W;
             static_for<0, r>([&](auto j_) {
                 constexpr int j = decltype(j_)::value;
@@ -99,8 +101,8 @@ __global__ void __launch_bounds__(C::THREADS, C::MINB) fourstep_pass2_kernel(con
             });
         });
     }
-    e.dif(sm, a.tw, t);
-    if (active) e.template store_last<TOut, INV>(a.out, b * a.dist_out + rg * W, a.n1, t, a.scale);
+    e.dif(sm, a.tw);
+    if (active) e.template store_last<TOut, INV>(a.out, b * a.dist_out + rg * W, a.n1, a.scale);
 }
 
 template <class C, bool INV, class TI, class TO, int PASS>
@@ -109,10 +111,7 @@ cudaError_t launch_fourstep(const FourStepArgs& a, cudaStream_t st) {
     auto kernel = (PASS == 1) ? fourstep_pass1_kernel<C, INV, TI, TO> : fourstep_pass2_kernel<C, INV, TI, TO>;
     cudaError_t e = ensure_smem(kernel, C::SMEM_BYTES, done);
     if (e != cudaSuccess) return e;
-    const int64_t grid = (a.tiles + C::G - 1) / C::G;
-    kernel<<<(unsigned)grid, C::THREADS, C::SMEM_BYTES, st>>>(a);
-    g_launch_count.fetch_add(1, std::memory_order_relaxed);
-    return cudaGetLastError();
+    return launch_tiles<C>(kernel, a, a.tiles, st);
 }
 
 template <class C, bool INV, class TS, int PASS>

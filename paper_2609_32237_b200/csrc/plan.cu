@@ -19,6 +19,7 @@ struct b200fft_plan_s {
     int direction, dtype;
     Layout layout;
     bool four_step;
+    int cluster;                 // CTAs per tile requested by the "cluster" option (0 = default)
     const KernelEntry* kernel;   // single-pass variant
     float2* tw;                  // its twiddle rows (device)
     int device;
@@ -33,9 +34,17 @@ static int elem_bytes(int dtype) { return dtype == B200FFT_C64 ? 8 : 4; }
 
 static int build_single_pass(b200fft_plan_s* p) {
     const bool inv = p->direction == B200FFT_INVERSE;
-    p->kernel = (p->layout == LAYOUT_ROWS) ? find_rows_kernel((int)p->n, inv, p->dtype, p->dtype)
-                                           : find_cols_kernel((int)p->n, inv, p->dtype, p->dtype);
-    if (!p->kernel) return B200FFT_ERR_UNSUPPORTED;
+    const KernelEntry* k = (p->layout == LAYOUT_ROWS)
+                               ? find_rows_kernel((int)p->n, inv, p->dtype, p->dtype, p->cluster)
+                               : find_cols_kernel((int)p->n, inv, p->dtype, p->dtype, p->cluster);
+    if (!k) return B200FFT_ERR_UNSUPPORTED;
+    if (p->kernel && p->kernel->tw_total == k->tw_total) {   // same factorisation: the table is reusable
+        p->kernel = k;
+        return B200FFT_OK;
+    }
+    p->kernel = k;
+    if (p->tw) cudaFree(p->tw);
+    p->tw = nullptr;
     if (cudaMalloc(&p->tw, sizeof(float2) * (size_t)p->kernel->tw_total) != cudaSuccess) {
         cudaGetLastError();
         return B200FFT_ERR_ALLOC;
@@ -110,6 +119,17 @@ extern "C" int fft_plan_set_option(fft_plan_t p, const char* key, int64_t value)
                 if (rc != B200FFT_OK) return rc;
             }
             p->four_step = false;
+        }
+        return B200FFT_OK;
+    }
+    if (std::strcmp(key, "cluster") == 0) {
+        if (p->four_step || p->n > 16384) return B200FFT_ERR_UNSUPPORTED;
+        const int old = p->cluster;
+        p->cluster = (int)value;
+        int rc = build_single_pass(p);
+        if (rc != B200FFT_OK) {
+            p->cluster = old;
+            return rc;
         }
         return B200FFT_OK;
     }

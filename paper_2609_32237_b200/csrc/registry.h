@@ -10,7 +10,7 @@ namespace b200fft {
 extern std::atomic<int64_t> g_launch_count;
 
 struct KernelEntry {
-    int n, w, g, threads, smem_bytes, tw_total;
+    int n, w, g, cl, threads, smem_bytes, tw_total;
     bool inverse;
     int in_dtype, out_dtype;                 // 0 = c64, 1 = c32h
     cudaError_t (*launch)(const FftArgs&, cudaStream_t);
@@ -32,15 +32,34 @@ inline cudaError_t ensure_smem(K kernel, int bytes, bool* done_per_device) {
     return cudaSuccess;
 }
 
+// Launch `kernel` over `tiles` tiles of configuration C: G tiles per CTA, or a
+// cluster of CL CTAs per tile.
+template <class C, class K, class A>
+cudaError_t launch_tiles(K kernel, const A& a, int64_t tiles, cudaStream_t st) {
+    const int64_t grid = (C::CL > 1) ? tiles * C::CL : (tiles + C::G - 1) / C::G;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid, 1, 1);
+    cfg.blockDim = dim3(C::THREADS, 1, 1);
+    cfg.dynamicSmemBytes = C::SMEM_BYTES;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = C::CL;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = (C::CL > 1) ? 1 : 0;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, a);
+    g_launch_count.fetch_add(1, std::memory_order_relaxed);
+    return e != cudaSuccess ? e : cudaGetLastError();
+}
+
 template <class C, bool INV, class TI, class TO>
 cudaError_t launch_fft(const FftArgs& a, cudaStream_t st) {
     static bool done[64] = {};
     cudaError_t e = ensure_smem(fft_kernel<C, INV, TI, TO>, C::SMEM_BYTES, done);
     if (e != cudaSuccess) return e;
-    const int64_t grid = (a.tiles + C::G - 1) / C::G;
-    fft_kernel<C, INV, TI, TO><<<(unsigned)grid, C::THREADS, C::SMEM_BYTES, st>>>(a);
-    g_launch_count.fetch_add(1, std::memory_order_relaxed);
-    return cudaGetLastError();
+    return launch_tiles<C>(fft_kernel<C, INV, TI, TO>, a, a.tiles, st);
 }
 
 template <class C>
@@ -52,7 +71,7 @@ cudaError_t launch_build_tw(float2* tw, cudaStream_t st) {
 
 template <class C, bool INV, class TI, class TO>
 constexpr KernelEntry make_entry() {
-    return KernelEntry{C::N, C::W, C::G, C::THREADS, C::SMEM_BYTES, C::TW_TOTAL, INV,
+    return KernelEntry{C::N, C::W, C::G, C::CL, C::THREADS, C::SMEM_BYTES, C::TW_TOTAL, INV,
                        TI::ELEM_BYTES == 8 ? 0 : 1, TO::ELEM_BYTES == 8 ? 0 : 1,
                        &launch_fft<C, INV, TI, TO>, &launch_build_tw<C>};
 }
@@ -64,7 +83,8 @@ constexpr KernelEntry make_entry() {
     make_entry<C, false, StoreC32H, StoreC32H>(),           \
     make_entry<C, true, StoreC32H, StoreC32H>()
 
-const KernelEntry* find_rows_kernel(int n, bool inverse, int in_dtype, int out_dtype);
-const KernelEntry* find_cols_kernel(int n, bool inverse, int in_dtype, int out_dtype);
+// cl: CTAs per tile (cluster size); 0 picks the default variant for that size
+const KernelEntry* find_rows_kernel(int n, bool inverse, int in_dtype, int out_dtype, int cl = 0);
+const KernelEntry* find_cols_kernel(int n, bool inverse, int in_dtype, int out_dtype, int cl = 0);
 
 }  // namespace b200fft

@@ -46,21 +46,23 @@ __global__ void __launch_bounds__(C::THREADS, C::MINB) sar_range_compress_kernel
     extern __shared__ __align__(16) float2 smem_dyn[];
     static_assert(C::W == 1, "range compression works on contiguous rows");
     const int g = threadIdx.x / C::T, t = threadIdx.x % C::T;
-    int64_t tile = (int64_t)blockIdx.x * C::G + g;
+    int64_t tile = (C::CL > 1) ? (int64_t)(blockIdx.x / C::CL) : (int64_t)blockIdx.x * C::G + g;
     const bool active = tile < a.tiles;
     if (!active) tile = a.tiles - 1;
-    float2* sm = smem_dyn + g * C::TILE_ELEMS;
+    float2* sm = smem_dyn + g * C::LOCAL_ELEMS;
     const int64_t base = tile * a.ld;
     Engine<C> e;
-    e.template load_first<StoreC64, false>(a.in, base, a.ld, t);
-    e.dif(sm, a.tw, t);
+    e.setup(t);
+    e.template load_first<StoreC64, false>(a.in, base, a.ld);
+    e.dif(sm, a.tw);
     {
         // registers hold X[b0 + KS j]; multiply by H at the same index, conjugate for the inverse
         using G = Geo<C, C::S>;
         constexpr int V = G::V, r = G::r, KS = C::N / r;
         static_for<0, V / 2>([&](auto h_) {
             constexpr int v = 2 * decltype(h_)::value;
-            const int b0 = V * t + v;
+            int b0, qq;
+            e.last_index(v, b0, qq);
             static_for<0, r>([&](auto j_) {
                 constexpr int j = decltype(j_)::value;
                 const float4 h = __ldg(reinterpret_cast<const float4*>(a.tab.H + j * KS + b0));
@@ -71,8 +73,8 @@ __global__ void __launch_bounds__(C::THREADS, C::MINB) sar_range_compress_kernel
             });
         });
     }
-    e.dit(sm, a.tw, t);
-    if (active) e.template store_first<TOut, true>(a.out, base, a.ld, t, 1.0f);
+    e.dit(sm, a.tw);
+    if (active) e.template store_first<TOut, true>(a.out, base, a.ld, 1.0f);
 }
 
 // ---------------------------------------------------------------- step 2
@@ -130,18 +132,19 @@ __global__ void __launch_bounds__(C::THREADS, C::MINB) sar_rcmc_filter_ifft_kern
     constexpr int W = C::W;
     static_assert(W >= 2, "azimuth transforms work on column tiles");
     const int g = threadIdx.x / C::T, t = threadIdx.x % C::T;
-    int64_t tile = (int64_t)blockIdx.x * C::G + g;
+    int64_t tile = (C::CL > 1) ? (int64_t)(blockIdx.x / C::CL) : (int64_t)blockIdx.x * C::G + g;
     const bool active = tile < a.tiles;
     if (!active) tile = a.tiles - 1;
-    float2* sm = smem_dyn + g * C::TILE_ELEMS;
+    float2* sm = smem_dyn + g * C::LOCAL_ELEMS;
     const int64_t base = tile * W;
     Engine<C> e;
+    e.setup(t);
     {
         using G = Geo<C, 1>;
         constexpr int V = G::V, r = G::r;
         static_for<0, V / 2>([&](auto h_) {
             constexpr int v = 2 * decltype(h_)::value;
-            const int c = V * t + v;
+            const int c = C::template cidx<V>(e.t, v, e.rank);
             const int q = c % W, lo = c / W;
             const int n0 = (int)base + q;                  // range bins n0, n0 + 1
             static_for<0, r>([&](auto j_) {
@@ -180,8 +183,8 @@ __global__ void __launch_bounds__(C::THREADS, C::MINB) sar_rcmc_filter_ifft_kern
             });
         });
     }
-    e.dif(sm, a.tw, t);
-    if (active) e.template store_last<StoreC64, true>(a.out, base, a.ld, t, a.scale);
+    e.dif(sm, a.tw);
+    if (active) e.template store_last<StoreC64, true>(a.out, base, a.ld, a.scale);
 }
 
 // ---------------------------------------------------------------- tables (float64, built once)
@@ -241,18 +244,14 @@ cudaError_t launch_range(const SarArgs& a, cudaStream_t st) {
     static bool done[64] = {};
     cudaError_t e = ensure_smem(sar_range_compress_kernel<C, TOut>, C::SMEM_BYTES, done);
     if (e != cudaSuccess) return e;
-    sar_range_compress_kernel<C, TOut><<<(unsigned)((a.tiles + C::G - 1) / C::G), C::THREADS, C::SMEM_BYTES, st>>>(a);
-    g_launch_count.fetch_add(1, std::memory_order_relaxed);
-    return cudaGetLastError();
+    return launch_tiles<C>(sar_range_compress_kernel<C, TOut>, a, a.tiles, st);
 }
 template <class C, class TIn>
 cudaError_t launch_rcmc(const SarArgs& a, cudaStream_t st) {
     static bool done[64] = {};
     cudaError_t e = ensure_smem(sar_rcmc_filter_ifft_kernel<C, TIn>, C::SMEM_BYTES, done);
     if (e != cudaSuccess) return e;
-    sar_rcmc_filter_ifft_kernel<C, TIn><<<(unsigned)((a.tiles + C::G - 1) / C::G), C::THREADS, C::SMEM_BYTES, st>>>(a);
-    g_launch_count.fetch_add(1, std::memory_order_relaxed);
-    return cudaGetLastError();
+    return launch_tiles<C>(sar_rcmc_filter_ifft_kernel<C, TIn>, a, a.tiles, st);
 }
 
 struct SarEntry {

@@ -116,6 +116,23 @@ def test_columns(n, cols, ld, direction):
         assert np.all(got[:, cols:] == 0)
 
 
+@pytest.mark.parametrize("n,cl", [(8192, 2), (8192, 4), (16384, 2), (16384, 4)])
+def test_rows_cluster_variants(n, cl):
+    """The same transform with a tile shared by a cluster of 2 or 4 CTAs (first
+    exchange through distributed shared memory): whole batch against the oracle."""
+    _check_rows(n, 5, seed=90 + cl, options={"cluster": cl})
+    _check_rows(n, 3, seed=91 + cl, direction=INV, gaussian=True, options={"cluster": cl})
+
+
+@pytest.mark.parametrize("n,cols,cl", [(2048, 8, 2), (4096, 12, 2), (4096, 12, 4), (8192, 6, 2)])
+def test_columns_cluster_variants(n, cols, cl):
+    m = inputs.uniform_complex64((n, cols), 33)
+    want = oracle.fft_cols(m.astype(np.complex128), FWD)
+    got = run_fft(to_device_c64(m), n, cols, cols, 1, FWD, C64, options={"cluster": cl}).cpu().numpy()
+    per_col = np.linalg.norm(got - want, axis=0) / np.linalg.norm(want, axis=0)
+    assert per_col.max() <= TOL32
+
+
 def test_columns_fp16_and_in_place():
     n, cols = 4096, 8
     m = inputs.uniform_complex64((n, cols), 31)
