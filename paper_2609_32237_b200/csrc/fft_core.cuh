@@ -316,6 +316,16 @@ struct StoreC64 {
         a = make_float2(v.x, v.y);
         b = make_float2(v.z, v.w);
     }
+    // the same load with a hint that L2 should bring in the whole 256-byte block on a miss:
+    // for column tiles, whose 32-byte row segments neighbour those of adjacent tiles
+    static __device__ __forceinline__ void load2_wide(const void* base, int64_t idx, float2& a, float2& b) {
+        float4 v;
+        asm volatile("ld.global.L2::256B.v4.f32 {%0, %1, %2, %3}, [%4];"
+                     : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w)
+                     : "l"(reinterpret_cast<const float2*>(base) + idx));
+        a = make_float2(v.x, v.y);
+        b = make_float2(v.z, v.w);
+    }
     static __device__ __forceinline__ void store2(void* base, int64_t idx, float2 a, float2 b) {
         *reinterpret_cast<float4*>(reinterpret_cast<float2*>(base) + idx) = make_float4(a.x, a.y, b.x, b.y);
     }
@@ -327,6 +337,14 @@ struct StoreC32H {
     static constexpr int ELEM_BYTES = 4;
     static __device__ __forceinline__ void load2(const void* base, int64_t idx, float2& a, float2& b) {
         const uint2 v = *reinterpret_cast<const uint2*>(reinterpret_cast<const __half2*>(base) + idx);
+        a = __half22float2(*reinterpret_cast<const __half2*>(&v.x));
+        b = __half22float2(*reinterpret_cast<const __half2*>(&v.y));
+    }
+    static __device__ __forceinline__ void load2_wide(const void* base, int64_t idx, float2& a, float2& b) {
+        uint2 v;
+        asm volatile("ld.global.L2::256B.v2.u32 {%0, %1}, [%2];"
+                     : "=r"(v.x), "=r"(v.y)
+                     : "l"(reinterpret_cast<const __half2*>(base) + idx));
         a = __half22float2(*reinterpret_cast<const __half2*>(&v.x));
         b = __half22float2(*reinterpret_cast<const __half2*>(&v.y));
     }
@@ -442,6 +460,9 @@ struct Engine {
             const float2* row = tw + C::tw_off(s) + lo0;
             static_for<1, r>([&](auto k_) {
                 constexpr int k = decltype(k_)::value;
+                // keep the compiler from hoisting all r-1 table loads above the arithmetic
+                // (that costs ~60 live registers on top of the 64 data registers)
+                if constexpr (DIT && (k % 4) == 1 && k > 1) asm volatile("" ::: "memory");
                 if constexpr (W == 1 && V >= 2) {
                     const float4 w = __ldg(reinterpret_cast<const float4*>(row + (k - 1) * Ls));
                     a[k] = cmul(a[k], make_float2(w.x, w.y));
@@ -501,7 +522,8 @@ struct Engine {
             static_for<0, r>([&](auto j_) {
                 constexpr int j = decltype(j_)::value;
                 const int64_t idx = (W == 1) ? base + j * G::Ls + lo : base + (int64_t)(j * G::Ls + lo) * ld + q;
-                ST::load2(in, idx, x[j * V + v], x[j * V + v + 1]);
+                if constexpr (W == 1) ST::load2(in, idx, x[j * V + v], x[j * V + v + 1]);
+                else ST::load2_wide(in, idx, x[j * V + v], x[j * V + v + 1]);
                 if constexpr (CONJ) {
                     x[j * V + v].y = -x[j * V + v].y;
                     x[j * V + v + 1].y = -x[j * V + v + 1].y;
@@ -576,6 +598,9 @@ struct Engine {
         static_assert(CL == 1, "the backward network is built for single-CTA tiles");
         static_for<0, S>([&](auto i_) {
             constexpr int s = S - decltype(i_)::value;
+            // Make the thread index opaque again at every stage: otherwise the compiler keeps
+            // the address arithmetic of the forward network alive for reuse here and spills.
+            asm volatile("" : "+r"(t));
             compute<s, true>(tw);
             if constexpr (s > 1) {
                 smem_rw<s, true>(sm);

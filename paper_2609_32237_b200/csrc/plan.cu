@@ -8,6 +8,7 @@
 
 namespace b200fft {
 std::atomic<int64_t> g_launch_count{0};
+int g_cosched = 1;
 }
 
 using namespace b200fft;
@@ -120,6 +121,11 @@ extern "C" int fft_plan_set_option(fft_plan_t p, const char* key, int64_t value)
             }
             p->four_step = false;
         }
+        return B200FFT_OK;
+    }
+    if (std::strcmp(key, "cosched") == 0) {
+        if (value < 1 || value > 16) return B200FFT_ERR_INVALID_ARG;
+        g_cosched = (int)value;
         return B200FFT_OK;
     }
     if (std::strcmp(key, "cluster") == 0) {

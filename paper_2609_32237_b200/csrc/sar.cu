@@ -27,6 +27,7 @@ struct SarTables {
     const float2* H;     // conj chirp spectrum / n_range, natural order, n_range entries
     const float4* mig;   // per Doppler bin: (g_hi, g_lo, a_frac, a_int as bits)
     const float4* phs;   // per Doppler bin: (A mod 1, B_hi, B_lo, 0)  [cycles]
+    const float2* stp;   // per Doppler bin: exp(j 2 pi B), the filter's step from one range bin to the next
 };
 
 struct SarArgs {
@@ -78,32 +79,6 @@ __global__ void __launch_bounds__(C::THREADS, C::MINB) sar_range_compress_kernel
 }
 
 // ---------------------------------------------------------------- step 2
-// weights of the 8-tap sinc interpolator, taps j = -3..4, unit sum:
-// sinc(mu - j) = (-1)^j sin(pi mu) / (pi (mu - j)); after normalisation the common
-// factor drops out, and multiplying through by prod_i (mu - i) removes the divisions:
-// w_j = (-1)^j P_j / sum_j' (-1)^j' P_j',  P_j = prod_{i != j} (mu - i).
-__device__ __forceinline__ void sinc8_weights(float mu, float (&w)[8]) {
-    float d[8], pre[8], suf[8];
-#pragma unroll
-    for (int i = 0; i < 8; ++i) d[i] = mu - (float)(i - 3);
-    pre[0] = 1.0f;
-#pragma unroll
-    for (int i = 1; i < 8; ++i) pre[i] = pre[i - 1] * d[i - 1];
-    suf[7] = 1.0f;
-#pragma unroll
-    for (int i = 6; i >= 0; --i) suf[i] = suf[i + 1] * d[i + 1];
-    float s = 0.0f;
-#pragma unroll
-    for (int i = 0; i < 8; ++i) {
-        const float p = pre[i] * suf[i];
-        w[i] = ((i - 3) & 1) ? -p : p;
-        s += w[i];
-    }
-    const float inv = 1.0f / s;
-#pragma unroll
-    for (int i = 0; i < 8; ++i) w[i] *= inv;
-}
-
 // Migration of (Doppler bin, range bin n): integer part and fraction, from the
 // per-bin slope split so that n * g_hi is exact in fp32.
 __device__ __forceinline__ void migration(const float4 m, int n, int& i0, float& mu) {
@@ -126,65 +101,174 @@ __device__ __forceinline__ float2 filter_phase(const float4 p, int n) {
     return make_float2(c, s);
 }
 
+// 16-byte asynchronous copy global -> shared, bypassing L1; `valid` false writes zeros
+// (samples outside the row read as zero).
+__device__ __forceinline__ void cp_async_16(void* smem_dst, const void* gmem_src, bool valid) {
+    const unsigned d = (unsigned)__cvta_generic_to_shared(smem_dst);
+    const int src = valid ? 16 : 0;
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(d), "l"(gmem_src), "r"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
+__device__ __forceinline__ float rcp_approx(float x) {
+    float r;
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x));
+    return r;
+}
+
+// weights of the 8-tap sinc interpolator, taps j = -3..4, unit sum:
+// sinc(mu - j) = (-1)^j sin(pi mu) / (pi (mu - j)); after normalisation the common factor
+// drops out: w_j = [(-1)^j / (mu - j)] / sum_j' [(-1)^j' / (mu - j')]. mu = 0 is nudged to
+// 1e-30, which gives w_0 = 1 and the others 1e-30: the exact limit to fp32 precision.
+__device__ __forceinline__ void sinc8_weights_rcp(float mu, float (&w)[8]) {
+    mu = fmaxf(mu, 1e-30f);
+    float s = 0.0f;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const float r = rcp_approx(mu - (float)(i - 3));
+        w[i] = ((i - 3) & 1) ? -r : r;
+        s += w[i];
+    }
+    const float inv = 1.0f / s;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) w[i] *= inv;
+}
+
+// The staged row windows live in the transform tile's own shared memory, which is idle
+// until the first exchange: 4 buffers of ROWS rows x 16 elements of the intermediate type.
 template <class C, class TIn>
-__global__ void __launch_bounds__(C::THREADS, C::MINB) sar_rcmc_filter_ifft_kernel(const SarArgs a) {
+constexpr int rcmc_smem_bytes() {
+    return C::SMEM_BYTES + C::N * 4;    // tile (doubles as staging) + one window start per row
+}
+
+template <class C, class TIn>
+__global__ void __launch_bounds__(C::THREADS, 1) sar_rcmc_filter_ifft_kernel(const SarArgs a) {
     extern __shared__ __align__(16) float2 smem_dyn[];
     constexpr int W = C::W;
-    static_assert(W >= 2, "azimuth transforms work on column tiles");
-    const int g = threadIdx.x / C::T, t = threadIdx.x % C::T;
-    int64_t tile = (C::CL > 1) ? (int64_t)(blockIdx.x / C::CL) : (int64_t)blockIdx.x * C::G + g;
-    const bool active = tile < a.tiles;
-    if (!active) tile = a.tiles - 1;
-    float2* sm = smem_dyn + g * C::LOCAL_ELEMS;
-    const int64_t base = tile * W;
+    static_assert(W == 4 && C::CL == 1 && C::G == 1 && C::radix(1) == 16, "column tiles of four range bins");
+    using G1 = Geo<C, 1>;
+    constexpr int V = G1::V, r = G1::r, ROWS = G1::Ls;          // ROWS Doppler bins per chunk, r chunks
+    static_assert(V == 2, "two adjacent range bins per thread");
+    constexpr int EB = TIn::ELEM_BYTES;
+    constexpr int WIN = 16;                                     // staged samples per row
+    constexpr int GRAN = 16 / EB;                               // samples per 16-byte copy
+    constexpr int NG = WIN / GRAN;                              // copies per row
+    constexpr int COPIES = ROWS * NG / C::THREADS;              // copies per thread per chunk
+    static_assert(ROWS * NG % C::THREADS == 0 && COPIES >= 1, "staging copies divide among threads");
+    static_assert(4 * ROWS * WIN * EB <= C::SMEM_BYTES, "four staging buffers fit in the tile");
+    using elem_t = typename std::conditional<EB == 8, float2, __half2>::type;
+
+    const int t = threadIdx.x;
+    const int64_t tile = blockIdx.x;
+    float2* sm = smem_dyn;
+    elem_t* stg = reinterpret_cast<elem_t*>(smem_dyn);
+    int* wstart = reinterpret_cast<int*>(smem_dyn + C::LOCAL_ELEMS);
+    const int n0 = (int)(tile * W);                              // first range bin of the tile
+    const elem_t* in = reinterpret_cast<const elem_t*>(a.in);
+
+    // window start of every Doppler bin of this tile: n0 + floor(migration at n0) - 3,
+    // rounded down to a 16-byte boundary
+    for (int k = t; k < C::N; k += C::THREADS) {
+        int i0;
+        float mu;
+        migration(__ldg(a.tab.mig + k), n0, i0, mu);
+        wstart[k] = (n0 + i0 - 3) & ~(GRAN - 1);
+    }
+    __syncthreads();
+
+    // element index of sample `smp` of row `row` in staging buffer `buf`: 16-byte granules
+    // are XOR-swizzled with the row so that rows read in parallel hit different banks
+    auto stg_index = [&](int buf, int row, int smp) {
+        return (buf * ROWS + row) * WIN + ((((smp / GRAN) ^ row) & (NG - 1)) * GRAN) + (smp % GRAN);
+    };
+    auto stage_chunk = [&](int j) {
+#pragma unroll
+        for (int i = 0; i < COPIES; ++i) {
+            const int idx = i * C::THREADS + t;
+            const int row = idx / NG, gr = idx % NG;
+            const int k = j * ROWS + row;
+            const int col = wstart[k] + gr * GRAN;
+            const bool valid = col >= 0 && col + GRAN <= a.nr;
+            cp_async_16(stg + stg_index(j & 3, row, gr * GRAN), in + (int64_t)k * a.ld + (valid ? col : 0), valid);
+        }
+    };
+
     Engine<C> e;
     e.setup(t);
-    {
-        using G = Geo<C, 1>;
-        constexpr int V = G::V, r = G::r;
-        static_for<0, V / 2>([&](auto h_) {
-            constexpr int v = 2 * decltype(h_)::value;
-            const int c = C::template cidx<V>(e.t, v, e.rank);
-            const int q = c % W, lo = c / W;
-            const int n0 = (int)base + q;                  // range bins n0, n0 + 1
-            static_for<0, r>([&](auto j_) {
-                constexpr int j = decltype(j_)::value;
-                const int k = j * G::Ls + lo;              // Doppler bin (row)
-                const float4 mg = __ldg(a.tab.mig + k);
-                const float4 ph = __ldg(a.tab.phs + k);
-                int ia, ib;
-                float mua, mub;
-                migration(mg, n0, ia, mua);
-                migration(mg, n0 + 1, ib, mub);
-                float wa[8], wb[8];
-                sinc8_weights(mua, wa);
-                sinc8_weights(mub, wb);
-                const int64_t row = (int64_t)k * a.ld;
-                float2 sa = make_float2(0.f, 0.f), sb = make_float2(0.f, 0.f);
+    const int c0 = C::template cidx<V>(t, 0, 0);
+    const int q = c0 % W, lo = c0 / W;                           // range bins n0+q, n0+q+1; row lo of each chunk
+
+    auto interp_chunk = [&](auto j_) {
+        constexpr int j = decltype(j_)::value;
+        const int k = j * ROWS + lo;                             // Doppler bin
+        const float4 mg = __ldg(a.tab.mig + k);
+        const float4 ph = __ldg(a.tab.phs + k);
+        int ia, ib;
+        float mua, mub;
+        migration(mg, n0 + q, ia, mua);
+        // one range bin on: the migration grows by the slope g = g_hi + g_lo
+        mub = mua + (mg.x + mg.y);
+        ib = ia;
+        if (mub >= 1.0f) {
+            mub -= 1.0f;
+            ib += 1;
+        }
+        float wa[8], wb[8];
+        sinc8_weights_rcp(mua, wa);
+        sinc8_weights_rcp(mub, wb);
+        const int ws = wstart[k];
+        // first tap (j = -3) of each bin, relative to the staged window
+        const int oa = min(max(n0 + q + ia - 3 - ws, 0), WIN - 8);
+        const int ob = min(max(n0 + q + 1 + ib - 3 - ws, 0), WIN - 8);
+        float2 sa = make_float2(0.f, 0.f), sb = make_float2(0.f, 0.f);
 #pragma unroll
-                for (int tap = 0; tap < 8; ++tap) {
-                    const int ca = n0 + ia + tap - 3, cb = n0 + 1 + ib + tap - 3;
-                    if (ca >= 0 && ca < a.nr) {
-                        const float2 s = TIn::load1(a.in, row + ca);
-                        sa.x = fmaf(wa[tap], s.x, sa.x);
-                        sa.y = fmaf(wa[tap], s.y, sa.y);
-                    }
-                    if (cb >= 0 && cb < a.nr) {
-                        const float2 s = TIn::load1(a.in, row + cb);
-                        sb.x = fmaf(wb[tap], s.x, sb.x);
-                        sb.y = fmaf(wb[tap], s.y, sb.y);
-                    }
-                }
-                const float2 fa = filter_phase(ph, n0), fb = filter_phase(ph, n0 + 1);
-                const float2 ya = cmul(sa, fa), yb = cmul(sb, fb);
-                // conjugate: the inverse transform is conj(FFT(conj(.)))
-                e.x[j * V + v] = make_float2(ya.x, -ya.y);
-                e.x[j * V + v + 1] = make_float2(yb.x, -yb.y);
-            });
-        });
-    }
+        for (int tap = 0; tap < 8; ++tap) {
+            float2 u, w2;
+            if constexpr (EB == 8) {
+                u = stg[stg_index(j & 3, lo, oa + tap)];
+                w2 = stg[stg_index(j & 3, lo, ob + tap)];
+            } else {
+                u = __half22float2(stg[stg_index(j & 3, lo, oa + tap)]);
+                w2 = __half22float2(stg[stg_index(j & 3, lo, ob + tap)]);
+            }
+            sa.x = fmaf(wa[tap], u.x, sa.x);
+            sa.y = fmaf(wa[tap], u.y, sa.y);
+            sb.x = fmaf(wb[tap], w2.x, sb.x);
+            sb.y = fmaf(wb[tap], w2.y, sb.y);
+        }
+        const float2 fa = filter_phase(ph, n0 + q);
+        const float2 fb = cmul(fa, __ldg(a.tab.stp + k));        // one more range bin: times exp(j 2 pi B)
+        const float2 ya = cmul(sa, fa), yb = cmul(sb, fb);
+        // conjugate: the inverse transform is conj(FFT(conj(.)))
+        e.x[j * V] = make_float2(ya.x, -ya.y);
+        e.x[j * V + 1] = make_float2(yb.x, -yb.y);
+    };
+
+    // two chunks per step; the pair two steps back has been consumed when its buffers are refilled
+    stage_chunk(0);
+    stage_chunk(1);
+    cp_async_commit();
+    stage_chunk(2);
+    stage_chunk(3);
+    cp_async_commit();
+    static_for<0, r / 2>([&](auto p_) {
+        constexpr int p = decltype(p_)::value;
+        if constexpr (p == 0) cp_async_wait<1>();
+        else cp_async_wait<0>();
+        __syncthreads();                       // pair p has landed for everyone; pair p-1 is consumed
+        if constexpr (p >= 1 && p + 1 < r / 2) {
+            stage_chunk(2 * p + 2);
+            stage_chunk(2 * p + 3);
+            cp_async_commit();
+        }
+        interp_chunk(IntC<2 * p>{});
+        interp_chunk(IntC<2 * p + 1>{});
+    });
+    __syncthreads();                           // staging is done with the tile buffer
     e.dif(sm, a.tw);
-    if (active) e.template store_last<StoreC64, true>(a.out, base, a.ld, a.scale);
+    e.template store_last<StoreC64, true>(a.out, (int64_t)n0, a.ld, a.scale);
 }
 
 // ---------------------------------------------------------------- tables (float64, built once)
@@ -214,7 +298,7 @@ __device__ double round_to_bits(double v, int bits) {
     return ldexp(rint(ldexp(m, bits)), ex - bits);
 }
 
-__global__ void sar_build_doppler_tables(float4* mig, float4* phs, int na, int nr, double wavelength,
+__global__ void sar_build_doppler_tables(float4* mig, float4* phs, float2* stp, int na, int nr, double wavelength,
                                          double prf, double velocity, double r_center, double dr) {
     const int k = blockIdx.x * blockDim.x + threadIdx.x;
     if (k >= na) return;
@@ -236,6 +320,9 @@ __global__ void sar_build_doppler_tables(float4* mig, float4* phs, int na, int n
     const double B = (2.0 * dr / wavelength) * d_minus_1;
     const double b_hi = round_to_bits(B, 10);
     phs[k] = make_float4((float)(A - floor(A)), (float)b_hi, (float)(B - b_hi), 0.0f);
+    double sn, cs;
+    sincospi(2.0 * (B - floor(B)), &sn, &cs);
+    stp[k] = make_float2((float)cs, (float)sn);
 }
 
 // ---------------------------------------------------------------- host side
@@ -249,9 +336,13 @@ cudaError_t launch_range(const SarArgs& a, cudaStream_t st) {
 template <class C, class TIn>
 cudaError_t launch_rcmc(const SarArgs& a, cudaStream_t st) {
     static bool done[64] = {};
-    cudaError_t e = ensure_smem(sar_rcmc_filter_ifft_kernel<C, TIn>, C::SMEM_BYTES, done);
+    constexpr int smem = rcmc_smem_bytes<C, TIn>();
+    static_assert(smem <= 227 * 1024, "tile + staging must fit one CTA's shared memory");
+    cudaError_t e = ensure_smem(sar_rcmc_filter_ifft_kernel<C, TIn>, smem, done);
     if (e != cudaSuccess) return e;
-    return launch_tiles<C>(sar_rcmc_filter_ifft_kernel<C, TIn>, a, a.tiles, st);
+    sar_rcmc_filter_ifft_kernel<C, TIn><<<(unsigned)a.tiles, C::THREADS, smem, st>>>(a);
+    g_launch_count.fetch_add(1, std::memory_order_relaxed);
+    return cudaGetLastError();
 }
 
 struct SarEntry {
@@ -286,6 +377,7 @@ struct b200fft_sar_s {
     const SarEntry* rcmc;
     float2 *tw_range, *tw_az, *H;
     float4 *mig, *phs;
+    float2* stp;
     void* workspace;
     size_t workspace_bytes;
 };
@@ -296,6 +388,7 @@ static void sar_release(b200fft_sar_s* p) {
     if (p->H) cudaFree(p->H);
     if (p->mig) cudaFree(p->mig);
     if (p->phs) cudaFree(p->phs);
+    if (p->stp) cudaFree(p->stp);
 }
 
 extern "C" int sar_rda_params_create(sar_rda_params_t* params, const sar_rda_desc* d) {
@@ -308,6 +401,10 @@ extern "C" int sar_rda_params_create(sar_rda_params_t* params, const sar_rda_des
     if (d->rcmc_taps != 8) return B200FFT_ERR_UNSUPPORTED;
     const double wavelength = kLight / d->carrier_hz;
     if (wavelength * d->prf_hz / (4.0 * d->velocity_mps) >= 0.5) return B200FFT_ERR_INVALID_ARG;  // D must stay real
+    {   // the staged window assumes the migration grows by less than one bin across four range bins
+        const double aa = wavelength * d->prf_hz / (4.0 * d->velocity_mps), u = aa * aa, sq = sqrt(1.0 - u);
+        if (4.0 * u / ((1.0 + sq) * sq) >= 1.0) return B200FFT_ERR_UNSUPPORTED;
+    }
     const long long pulse_samples = llround(d->pulse_s * d->fs_hz);
     if (pulse_samples < 1 || pulse_samples > d->n_range) return B200FFT_ERR_INVALID_ARG;
 
@@ -326,7 +423,8 @@ extern "C" int sar_rda_params_create(sar_rda_params_t* params, const sar_rda_des
               cudaMalloc(&p->tw_az, sizeof(float2) * (size_t)p->rcmc->tw_total) == cudaSuccess &&
               cudaMalloc(&p->H, sizeof(float2) * (size_t)nr) == cudaSuccess &&
               cudaMalloc(&p->mig, sizeof(float4) * (size_t)na) == cudaSuccess &&
-              cudaMalloc(&p->phs, sizeof(float4) * (size_t)na) == cudaSuccess;
+              cudaMalloc(&p->phs, sizeof(float4) * (size_t)na) == cudaSuccess &&
+              cudaMalloc(&p->stp, sizeof(float2) * (size_t)na) == cudaSuccess;
     if (!ok) {
         cudaGetLastError();
         sar_release(p);
@@ -337,7 +435,7 @@ extern "C" int sar_rda_params_create(sar_rda_params_t* params, const sar_rda_des
     const double kappa = (d->bandwidth_hz / d->pulse_s) / (d->fs_hz * d->fs_hz);
     ok = p->range->build_tw(p->tw_range, 0) == cudaSuccess && p->rcmc->build_tw(p->tw_az, 0) == cudaSuccess;
     sar_build_matched_filter<<<(nr + 127) / 128, 128>>>(p->H, nr, (int)pulse_samples, kappa);
-    sar_build_doppler_tables<<<(na + 127) / 128, 128>>>(p->mig, p->phs, na, nr, wavelength, d->prf_hz,
+    sar_build_doppler_tables<<<(na + 127) / 128, 128>>>(p->mig, p->phs, p->stp, na, nr, wavelength, d->prf_hz,
                                                        d->velocity_mps, d->r_center_m, dr);
     g_launch_count.fetch_add(2, std::memory_order_relaxed);
     ok = ok && cudaGetLastError() == cudaSuccess && cudaStreamSynchronize(0) == cudaSuccess;
@@ -377,7 +475,7 @@ extern "C" int sar_rda_run_step(const void* raw, sar_rda_params_t p, void* out, 
         if (reinterpret_cast<uintptr_t>(raw) % 16) return B200FFT_ERR_ALIGNMENT;
         SarArgs a{};
         a.in = raw; a.out = p->workspace; a.tw = p->tw_range;
-        a.tab = SarTables{p->H, p->mig, p->phs};
+        a.tab = SarTables{p->H, p->mig, p->phs, p->stp};
         a.tiles = na; a.ld = nr; a.nr = (int)nr; a.scale = 1.0f;
         return p->range->launch(a, st) == cudaSuccess ? B200FFT_OK : B200FFT_ERR_CUDA;
     }
@@ -392,7 +490,7 @@ extern "C" int sar_rda_run_step(const void* raw, sar_rda_params_t p, void* out, 
     if (reinterpret_cast<uintptr_t>(out) % 16) return B200FFT_ERR_ALIGNMENT;
     SarArgs a{};
     a.in = p->workspace; a.out = out; a.tw = p->tw_az;
-    a.tab = SarTables{p->H, p->mig, p->phs};
+    a.tab = SarTables{p->H, p->mig, p->phs, p->stp};
     a.tiles = nr / p->rcmc->w; a.ld = nr; a.nr = (int)nr; a.scale = 1.0f;
     return p->rcmc->launch(a, st) == cudaSuccess ? B200FFT_OK : B200FFT_ERR_CUDA;
 }
