@@ -100,7 +100,9 @@ int fft_plan_destroy(fft_plan_t plan);
  * "cluster" value c (1, 2 or 4; 0 = the default for that size) picks the
  * variant of a single-pass plan in which c CTAs of one thread-block cluster
  * share a tile through distributed shared memory; B200FFT_ERR_UNSUPPORTED if
- * that variant is not compiled for the plan's size. Unknown keys return
+ * that variant is not compiled for the plan's size. Key "prefetch" value d
+ * makes each CTA of a rows plan ask L2 for the input of the transform d tiles
+ * ahead (0 = off, -1 = the default: one wave ahead for n = 16384). Unknown keys return
  * B200FFT_ERR_INVALID_ARG. Must be called before set_workspace. */
 int fft_plan_set_option(fft_plan_t plan, const char *key, int64_t value);
 

@@ -32,7 +32,6 @@ using T8192 = Cfg<8192, 2, 32, 1, 1, 16, 32, 16>;
 using T2048x2 = Cfg<2048, 4, 32, 1, 2, 16, 8, 16>;
 using T4096x2 = Cfg<4096, 4, 32, 1, 2, 16, 16, 16>;
 using T4096x4 = Cfg<4096, 4, 32, 1, 4, 16, 16, 16>;
-using T4096w2 = Cfg<4096, 2, 32, 1, 1, 16, 16, 16>;
 using T8192x2 = Cfg<8192, 2, 32, 1, 2, 16, 32, 16>;
 
 }  // namespace b200fft

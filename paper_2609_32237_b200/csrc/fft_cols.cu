@@ -9,17 +9,15 @@ static const KernelEntry k_cols[] = {
     B200FFT_ENTRIES_STD(T256),  B200FFT_ENTRIES_STD(T512),  B200FFT_ENTRIES_STD(T1024),
     B200FFT_ENTRIES_STD(T2048), B200FFT_ENTRIES_STD(T4096), B200FFT_ENTRIES_STD(T8192),
     B200FFT_ENTRIES_STD(T2048x2), B200FFT_ENTRIES_STD(T4096x2), B200FFT_ENTRIES_STD(T4096x4),
-    B200FFT_ENTRIES_STD(T8192x2), B200FFT_ENTRIES_STD(T4096w2),
+    B200FFT_ENTRIES_STD(T8192x2),
 };
 
 static int default_cluster(int n) { return 1; }
 
 const KernelEntry* find_cols_kernel(int n, bool inverse, int in_dtype, int out_dtype, int cl) {
-    int w = 0;
-    if (cl >= 100) { w = cl / 100; cl %= 100; }      // tuning: cl = 100 * width + cluster
     if (cl == 0) cl = default_cluster(n);
     for (const KernelEntry& e : k_cols)
-        if (e.n == n && e.cl == cl && (w == 0 || e.w == w) && e.inverse == inverse && e.in_dtype == in_dtype && e.out_dtype == out_dtype) return &e;
+        if (e.n == n && e.cl == cl && e.inverse == inverse && e.in_dtype == in_dtype && e.out_dtype == out_dtype) return &e;
     return nullptr;
 }
 

@@ -316,35 +316,20 @@ struct StoreC64 {
         a = make_float2(v.x, v.y);
         b = make_float2(v.z, v.w);
     }
-    // the same load with a hint that L2 should bring in the whole 256-byte block on a miss:
-    // for column tiles, whose 32-byte row segments neighbour those of adjacent tiles
-    static __device__ __forceinline__ void load2_wide(const void* base, int64_t idx, float2& a, float2& b) {
-        float4 v;
-        asm volatile("ld.global.L2::256B.v4.f32 {%0, %1, %2, %3}, [%4];"
-                     : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w)
-                     : "l"(reinterpret_cast<const float2*>(base) + idx));
-        a = make_float2(v.x, v.y);
-        b = make_float2(v.z, v.w);
-    }
     static __device__ __forceinline__ void store2(void* base, int64_t idx, float2 a, float2 b) {
         *reinterpret_cast<float4*>(reinterpret_cast<float2*>(base) + idx) = make_float4(a.x, a.y, b.x, b.y);
     }
     static __device__ __forceinline__ float2 load1(const void* base, int64_t idx) {
         return reinterpret_cast<const float2*>(base)[idx];
     }
+    static __device__ __forceinline__ void store1(void* base, int64_t idx, float2 a) {
+        reinterpret_cast<float2*>(base)[idx] = a;
+    }
 };
 struct StoreC32H {
     static constexpr int ELEM_BYTES = 4;
     static __device__ __forceinline__ void load2(const void* base, int64_t idx, float2& a, float2& b) {
         const uint2 v = *reinterpret_cast<const uint2*>(reinterpret_cast<const __half2*>(base) + idx);
-        a = __half22float2(*reinterpret_cast<const __half2*>(&v.x));
-        b = __half22float2(*reinterpret_cast<const __half2*>(&v.y));
-    }
-    static __device__ __forceinline__ void load2_wide(const void* base, int64_t idx, float2& a, float2& b) {
-        uint2 v;
-        asm volatile("ld.global.L2::256B.v2.u32 {%0, %1}, [%2];"
-                     : "=r"(v.x), "=r"(v.y)
-                     : "l"(reinterpret_cast<const __half2*>(base) + idx));
         a = __half22float2(*reinterpret_cast<const __half2*>(&v.x));
         b = __half22float2(*reinterpret_cast<const __half2*>(&v.y));
     }
@@ -357,6 +342,9 @@ struct StoreC32H {
     }
     static __device__ __forceinline__ float2 load1(const void* base, int64_t idx) {
         return __half22float2(reinterpret_cast<const __half2*>(base)[idx]);
+    }
+    static __device__ __forceinline__ void store1(void* base, int64_t idx, float2 a) {
+        reinterpret_cast<__half2*>(base)[idx] = __float22half2_rn(a);
     }
 };
 
@@ -522,8 +510,7 @@ struct Engine {
             static_for<0, r>([&](auto j_) {
                 constexpr int j = decltype(j_)::value;
                 const int64_t idx = (W == 1) ? base + j * G::Ls + lo : base + (int64_t)(j * G::Ls + lo) * ld + q;
-                if constexpr (W == 1) ST::load2(in, idx, x[j * V + v], x[j * V + v + 1]);
-                else ST::load2_wide(in, idx, x[j * V + v], x[j * V + v + 1]);
+                ST::load2(in, idx, x[j * V + v], x[j * V + v + 1]);
                 if constexpr (CONJ) {
                     x[j * V + v].y = -x[j * V + v].y;
                     x[j * V + v + 1].y = -x[j * V + v + 1].y;
@@ -618,7 +605,13 @@ struct FftArgs {
     int64_t tiles;   // rows: batch; columns: batch / W
     int64_t dist;    // rows: elements between transforms; columns: elements between rows (ld)
     float scale;
+    int prefetch_ahead;   // rows: tiles ahead whose input one thread asks L2 to fetch (0 = off)
 };
+
+// Ask L2 to start fetching `bytes` contiguous bytes (a multiple of 16, 16-byte aligned).
+__device__ __forceinline__ void prefetch_l2_bulk(const void* p, unsigned bytes) {
+    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(p), "r"(bytes) : "memory");
+}
 
 // One CTA = G tiles, or one cluster of CL CTAs = one tile. INV: inverse via
 // conj(FFT(conj(x))) * scale.
@@ -633,6 +626,14 @@ __global__ void __launch_bounds__(C::THREADS, C::MINB) fft_kernel(const FftArgs 
     const int64_t base = (C::W == 1) ? tile * a.dist : tile * C::W;
     Engine<C> e;
     e.setup(t);
+    if constexpr (C::W == 1 && C::CL == 1 && C::G == 1) {
+        // A large tile leaves room for one or two CTAs per SM, so nothing overlaps this CTA's
+        // load phase. One thread asks L2 for the input of the tile that will run where this
+        // one runs now, some CTAs later; that tile's loads then hit L2.
+        if (a.prefetch_ahead > 0 && threadIdx.x == 0 && tile + a.prefetch_ahead < a.tiles)
+            prefetch_l2_bulk(reinterpret_cast<const char*>(a.in) + (tile + a.prefetch_ahead) * a.dist * TIn::ELEM_BYTES,
+                             (unsigned)(C::N * TIn::ELEM_BYTES));
+    }
     e.template load_first<TIn, INV>(a.in, base, a.dist);
     e.dif(sm, a.tw);
     if (active) e.template store_last<TOut, INV>(a.out, base, a.dist, a.scale);

@@ -8,7 +8,6 @@
 
 namespace b200fft {
 std::atomic<int64_t> g_launch_count{0};
-int g_cosched = 1;
 }
 
 using namespace b200fft;
@@ -21,9 +20,11 @@ struct b200fft_plan_s {
     Layout layout;
     bool four_step;
     int cluster;                 // CTAs per tile requested by the "cluster" option (0 = default)
+    int prefetch_ahead;          // "prefetch" option: tiles ahead to prefetch into L2 (-1 = default)
     const KernelEntry* kernel;   // single-pass variant
     float2* tw;                  // its twiddle rows (device)
     int device;
+    int sms;                     // multiprocessors of that device
     FourStep fs;                 // two-pass variant
     void* workspace;
     size_t workspace_bytes;
@@ -84,7 +85,10 @@ extern "C" int fft_plan_create(fft_plan_t* plan, int64_t n, int64_t batch, int64
     if (!p) return B200FFT_ERR_ALLOC;
     p->n = n; p->batch = batch; p->stride = stride; p->dist = dist;
     p->direction = direction; p->dtype = storage_dtype; p->layout = layout;
+    p->prefetch_ahead = -1;
     if (cudaGetDevice(&p->device) != cudaSuccess) { delete p; return B200FFT_ERR_CUDA; }
+    p->sms = 148;
+    cudaDeviceGetAttribute(&p->sms, cudaDevAttrMultiProcessorCount, p->device);
 
     int rc;
     if (n > 16384) {
@@ -123,9 +127,9 @@ extern "C" int fft_plan_set_option(fft_plan_t p, const char* key, int64_t value)
         }
         return B200FFT_OK;
     }
-    if (std::strcmp(key, "cosched") == 0) {
-        if (value < 1 || value > 16) return B200FFT_ERR_INVALID_ARG;
-        g_cosched = (int)value;
+    if (std::strcmp(key, "prefetch") == 0) {
+        if (value < -1 || value > (1 << 20)) return B200FFT_ERR_INVALID_ARG;
+        p->prefetch_ahead = (int)value;
         return B200FFT_OK;
     }
     if (std::strcmp(key, "cluster") == 0) {
@@ -175,6 +179,14 @@ extern "C" int fft_execute(fft_plan_t p, const void* in, void* out, void* stream
     a.in = in;
     a.out = out;
     a.tw = p->tw;
+    a.prefetch_ahead = 0;
+    if (p->layout == LAYOUT_ROWS && p->kernel->cl == 1 && p->kernel->g == 1) {
+        // default: for tiles that fill an SM (one CTA resident), the tile one full wave ahead;
+        // measured on B200: +13 % at n = 16384 rows, nothing to gain at n = 8192 and below,
+        // and a loss for column tiles (their time goes to the lock-step compute, not the load)
+        const bool fills_sm = p->kernel->smem_bytes > 100 * 1024;
+        a.prefetch_ahead = (p->prefetch_ahead >= 0) ? p->prefetch_ahead : (fills_sm ? p->sms : 0);
+    }
     a.scale = (p->direction == B200FFT_INVERSE) ? (float)(1.0 / (double)p->n) : 1.0f;
     if (p->layout == LAYOUT_ROWS) {
         a.tiles = p->batch;

@@ -8,9 +8,6 @@
 namespace b200fft {
 
 extern std::atomic<int64_t> g_launch_count;
-// tuning knob: launch single-CTA tiles in clusters of this many CTAs (adjacent tiles are then
-// co-scheduled on one GPC); 1 = plain launch
-extern int g_cosched;
 
 struct KernelEntry {
     int n, w, g, cl, threads, smem_bytes, tw_total;
@@ -50,9 +47,8 @@ cudaError_t launch_tiles(K kernel, const A& a, int64_t tiles, cudaStream_t st) {
     attr[0].val.clusterDim.x = C::CL;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
-    if (C::CL == 1 && g_cosched > 1 && grid % g_cosched == 0) attr[0].val.clusterDim.x = g_cosched;
     cfg.attrs = attr;
-    cfg.numAttrs = (attr[0].val.clusterDim.x > 1) ? 1 : 0;
+    cfg.numAttrs = (C::CL > 1) ? 1 : 0;
     cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, a);
     g_launch_count.fetch_add(1, std::memory_order_relaxed);
     return e != cudaSuccess ? e : cudaGetLastError();

@@ -96,8 +96,12 @@ __device__ __forceinline__ float2 filter_phase(const float4 p, int n) {
     const float fn = (float)n;
     const float t = fn * p.y;
     const float f = (t - floorf(t)) + fmaf(fn, p.z, p.x);
+    // fraction of a cycle in [-0.5, 0.5): the hardware sine/cosine are accurate to about
+    // 4e-7 absolute on [-pi, pi], well inside the error budget of the fp32 chain
+    float fr = f - floorf(f);
+    fr = (fr >= 0.5f) ? fr - 1.0f : fr;
     float s, c;
-    sincospif(2.0f * (f - floorf(f)), &s, &c);
+    __sincosf(6.283185307179586f * fr, &s, &c);
     return make_float2(c, s);
 }
 
@@ -120,27 +124,36 @@ __device__ __forceinline__ float rcp_approx(float x) {
 
 // weights of the 8-tap sinc interpolator, taps j = -3..4, unit sum:
 // sinc(mu - j) = (-1)^j sin(pi mu) / (pi (mu - j)); after normalisation the common factor
-// drops out: w_j = [(-1)^j / (mu - j)] / sum_j' [(-1)^j' / (mu - j')]. mu = 0 is nudged to
-// 1e-30, which gives w_0 = 1 and the others 1e-30: the exact limit to fp32 precision.
+// drops out: w_j = [(-1)^j / (mu - j)] / sum_j' [(-1)^j' / (mu - j')]. This returns the
+// magnitudes m_i = |1 / (mu - j)| * inv with the sign (-1)^j left to the caller (tap i = j + 3
+// is negative for even i). mu = 0 is nudged to 1e-30, which gives w_0 = 1 and the others
+// 1e-30: the exact limit to fp32 precision.
 __device__ __forceinline__ void sinc8_weights_rcp(float mu, float (&w)[8]) {
     mu = fmaxf(mu, 1e-30f);
     float s = 0.0f;
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
-        const float r = rcp_approx(mu - (float)(i - 3));
-        w[i] = ((i - 3) & 1) ? -r : r;
-        s += w[i];
+        w[i] = rcp_approx(mu - (float)(i - 3));     // sign (-1)^(i-3) applied below and by the caller
+        s = ((i - 3) & 1) ? s - w[i] : s + w[i];
     }
-    const float inv = 1.0f / s;
+    float inv = rcp_approx(s);
+    inv = inv * (2.0f - s * inv);                    // one Newton step: full fp32 accuracy
 #pragma unroll
     for (int i = 0; i < 8; ++i) w[i] *= inv;
 }
 
-// The staged row windows live in the transform tile's own shared memory, which is idle
-// until the first exchange: 4 buffers of ROWS rows x 16 elements of the intermediate type.
+// The staged row windows share the transform tile's shared memory, which is idle until
+// the first exchange: 4 buffers of ROWS rows, 16 elements of the intermediate type each
+// at a pitch of 16 + 16 bytes' worth (an odd number of 16-byte granules, so rows read
+// in parallel start in different banks).
 template <class C, class TIn>
-constexpr int rcmc_smem_bytes() {
-    return C::SMEM_BYTES + C::N * 4;    // tile (doubles as staging) + one window start per row
+__host__ __device__ constexpr int rcmc_pitch() { return 16 + 16 / TIn::ELEM_BYTES; }
+template <class C, class TIn>
+__host__ __device__ constexpr int rcmc_stage_bytes() { return 4 * (C::N / 16) * rcmc_pitch<C, TIn>() * TIn::ELEM_BYTES; }
+template <class C, class TIn>
+__host__ __device__ constexpr int rcmc_smem_bytes() {
+    constexpr int st = rcmc_stage_bytes<C, TIn>();
+    return (st > C::SMEM_BYTES ? st : C::SMEM_BYTES) + C::N * 4;   // + one window start per row
 }
 
 template <class C, class TIn>
@@ -157,14 +170,15 @@ __global__ void __launch_bounds__(C::THREADS, 1) sar_rcmc_filter_ifft_kernel(con
     constexpr int NG = WIN / GRAN;                              // copies per row
     constexpr int COPIES = ROWS * NG / C::THREADS;              // copies per thread per chunk
     static_assert(ROWS * NG % C::THREADS == 0 && COPIES >= 1, "staging copies divide among threads");
-    static_assert(4 * ROWS * WIN * EB <= C::SMEM_BYTES, "four staging buffers fit in the tile");
+    constexpr int PITCH = rcmc_pitch<C, TIn>();
+    constexpr int REGION = (rcmc_stage_bytes<C, TIn>() > C::SMEM_BYTES ? rcmc_stage_bytes<C, TIn>() : C::SMEM_BYTES);
     using elem_t = typename std::conditional<EB == 8, float2, __half2>::type;
 
     const int t = threadIdx.x;
     const int64_t tile = blockIdx.x;
     float2* sm = smem_dyn;
     elem_t* stg = reinterpret_cast<elem_t*>(smem_dyn);
-    int* wstart = reinterpret_cast<int*>(smem_dyn + C::LOCAL_ELEMS);
+    int* wstart = reinterpret_cast<int*>(reinterpret_cast<char*>(smem_dyn) + REGION);
     const int n0 = (int)(tile * W);                              // first range bin of the tile
     const elem_t* in = reinterpret_cast<const elem_t*>(a.in);
 
@@ -178,11 +192,7 @@ __global__ void __launch_bounds__(C::THREADS, 1) sar_rcmc_filter_ifft_kernel(con
     }
     __syncthreads();
 
-    // element index of sample `smp` of row `row` in staging buffer `buf`: 16-byte granules
-    // are XOR-swizzled with the row so that rows read in parallel hit different banks
-    auto stg_index = [&](int buf, int row, int smp) {
-        return (buf * ROWS + row) * WIN + ((((smp / GRAN) ^ row) & (NG - 1)) * GRAN) + (smp % GRAN);
-    };
+    auto stg_index = [&](int buf, int row, int smp) { return (buf * ROWS + row) * PITCH + smp; };
     auto stage_chunk = [&](int j) {
 #pragma unroll
         for (int i = 0; i < COPIES; ++i) {
@@ -223,20 +233,29 @@ __global__ void __launch_bounds__(C::THREADS, 1) sar_rcmc_filter_ifft_kernel(con
         const int oa = min(max(n0 + q + ia - 3 - ws, 0), WIN - 8);
         const int ob = min(max(n0 + q + 1 + ib - 3 - ws, 0), WIN - 8);
         float2 sa = make_float2(0.f, 0.f), sb = make_float2(0.f, 0.f);
+        const elem_t* pa = stg + stg_index(j & 3, lo, oa);
+        const elem_t* pb = stg + stg_index(j & 3, lo, ob);
 #pragma unroll
         for (int tap = 0; tap < 8; ++tap) {
             float2 u, w2;
             if constexpr (EB == 8) {
-                u = stg[stg_index(j & 3, lo, oa + tap)];
-                w2 = stg[stg_index(j & 3, lo, ob + tap)];
+                u = pa[tap];
+                w2 = pb[tap];
             } else {
-                u = __half22float2(stg[stg_index(j & 3, lo, oa + tap)]);
-                w2 = __half22float2(stg[stg_index(j & 3, lo, ob + tap)]);
+                u = __half22float2(pa[tap]);
+                w2 = __half22float2(pb[tap]);
             }
-            sa.x = fmaf(wa[tap], u.x, sa.x);
-            sa.y = fmaf(wa[tap], u.y, sa.y);
-            sb.x = fmaf(wb[tap], w2.x, sb.x);
-            sb.y = fmaf(wb[tap], w2.y, sb.y);
+            if ((tap - 3) & 1) {                                  // odd tap: weight is -|w|
+                sa.x = fmaf(-wa[tap], u.x, sa.x);
+                sa.y = fmaf(-wa[tap], u.y, sa.y);
+                sb.x = fmaf(-wb[tap], w2.x, sb.x);
+                sb.y = fmaf(-wb[tap], w2.y, sb.y);
+            } else {
+                sa.x = fmaf(wa[tap], u.x, sa.x);
+                sa.y = fmaf(wa[tap], u.y, sa.y);
+                sb.x = fmaf(wb[tap], w2.x, sb.x);
+                sb.y = fmaf(wb[tap], w2.y, sb.y);
+            }
         }
         const float2 fa = filter_phase(ph, n0 + q);
         const float2 fb = cmul(fa, __ldg(a.tab.stp + k));        // one more range bin: times exp(j 2 pi B)
@@ -484,6 +503,7 @@ extern "C" int sar_rda_run_step(const void* raw, sar_rda_params_t p, void* out, 
         a.in = p->workspace; a.out = p->workspace; a.tw = p->tw_az;
         a.tiles = nr / p->azfft->w; a.dist = nr;
         a.scale = (float)(1.0 / (double)na);
+        a.prefetch_ahead = 0;
         return p->azfft->launch(a, st) == cudaSuccess ? B200FFT_OK : B200FFT_ERR_CUDA;
     }
     if (!out) return B200FFT_ERR_INVALID_ARG;

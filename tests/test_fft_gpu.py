@@ -257,3 +257,4 @@ def test_config1_full_size_forward_and_inverse():
 def test_config2_full_size(n, batch, dtype):
     """N = 8192 x 16384 and N = 16384 x 8192, Gaussian, seed 2, fp32 and fp16 storage."""
     _sampled_full_size(n, batch, 2, dtype, FWD)
+
