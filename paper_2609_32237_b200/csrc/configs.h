@@ -19,6 +19,8 @@ using R8192x2 = Cfg<8192, 1, 32, 1, 2, 16, 32, 16>;
 using R8192x4 = Cfg<8192, 1, 32, 1, 4, 16, 32, 16>;
 using R16384x2 = Cfg<16384, 1, 32, 1, 2, 16, 4, 16, 16>;
 using R16384x4 = Cfg<16384, 1, 32, 1, 4, 16, 4, 16, 16>;
+// the same with every first-stage twiddle row loaded from the table instead of computed
+using R4096t15 = Cfg<4096, 1, 32, 1, 1, 16, 16, 16, 1, 15>;
 
 // W adjacent columns (or rows, in the second pass of the two-pass split) per tile
 using T64 = Cfg<64, 4, 32, 16, 1, 16, 4>;

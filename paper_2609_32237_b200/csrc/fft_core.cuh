@@ -161,9 +161,10 @@ struct Dft<32> {
 };
 
 // ------------------------------------------------------------ configuration
-template <int N_, int W_, int P_, int G_, int CL_, int R1_, int R2_, int R3_ = 1, int R4_ = 1>
+template <int N_, int W_, int P_, int G_, int CL_, int R1_, int R2_, int R3_ = 1, int R4_ = 1, int TW1_ = 1>
 struct Cfg {
     static constexpr int N = N_, W = W_, P = P_, G = G_, CL = CL_;
+    static constexpr int TW1_LOADS = TW1_;    // first-stage twiddle rows loaded from the table (rest computed)
     static constexpr int S = (R3_ == 1) ? 2 : ((R4_ == 1) ? 3 : 4);
     __host__ __device__ static constexpr int radix(int s) { return s == 1 ? R1_ : (s == 2 ? R2_ : (s == 3 ? R3_ : R4_)); }
     __host__ __device__ static constexpr int L(int s) {
@@ -443,24 +444,46 @@ struct Engine {
         using G = Geo<C, s>;
         constexpr int V = G::V, r = G::r, Ls = G::Ls;
         constexpr bool has_tw = !G::last;
+        // Rows of the stage's twiddle table that are loaded; the rest are products of loaded
+        // ones (w^k = w^M w^(k-M)). Only the first stage of a one-transform tile trades
+        // loads for arithmetic: there every lane needs different entries, so each table row
+        // costs four L1 wavefronts per warp, and L1 is the busiest unit of these kernels.
+        constexpr int M = (s == 1 && W == 1 && V >= 2 && r > C::TW1_LOADS) ? C::TW1_LOADS : r - 1;
         auto twiddle_pair = [&](int lo0, float2* a, float2* b) {
             // a, b: the r values of butterflies v, v+1 (b == nullptr if V == 1)
             const float2* row = tw + C::tw_off(s) + lo0;
-            static_for<1, r>([&](auto k_) {
-                constexpr int k = decltype(k_)::value;
-                // keep the compiler from hoisting all r-1 table loads above the arithmetic
-                // (that costs ~60 live registers on top of the 64 data registers)
-                if constexpr (DIT && (k % 4) == 1 && k > 1) asm volatile("" ::: "memory");
-                if constexpr (W == 1 && V >= 2) {
-                    const float4 w = __ldg(reinterpret_cast<const float4*>(row + (k - 1) * Ls));
-                    a[k] = cmul(a[k], make_float2(w.x, w.y));
-                    b[k] = cmul(b[k], make_float2(w.z, w.w));
-                } else {
-                    const float2 w = __ldg(row + (k - 1) * Ls);
-                    a[k] = cmul(a[k], w);
-                    if (b) b[k] = cmul(b[k], w);
-                }
-            });
+            if constexpr (M < r - 1) {
+                float2 wa[r], wb[r];
+                static_for<1, r>([&](auto k_) {
+                    constexpr int k = decltype(k_)::value;
+                    if constexpr (k <= M) {
+                        const float4 w = __ldg(reinterpret_cast<const float4*>(row + (k - 1) * Ls));
+                        wa[k] = make_float2(w.x, w.y);
+                        wb[k] = make_float2(w.z, w.w);
+                    } else {
+                        wa[k] = cmul(wa[M], wa[k - M]);
+                        wb[k] = cmul(wb[M], wb[k - M]);
+                    }
+                    a[k] = cmul(a[k], wa[k]);
+                    b[k] = cmul(b[k], wb[k]);
+                });
+            } else {
+                static_for<1, r>([&](auto k_) {
+                    constexpr int k = decltype(k_)::value;
+                    // keep the compiler from hoisting all r-1 table loads above the arithmetic
+                    // (that costs ~60 live registers on top of the 64 data registers)
+                    if constexpr (DIT && (k % 4) == 1 && k > 1) asm volatile("" ::: "memory");
+                    if constexpr (W == 1 && V >= 2) {
+                        const float4 w = __ldg(reinterpret_cast<const float4*>(row + (k - 1) * Ls));
+                        a[k] = cmul(a[k], make_float2(w.x, w.y));
+                        b[k] = cmul(b[k], make_float2(w.z, w.w));
+                    } else {
+                        const float2 w = __ldg(row + (k - 1) * Ls);
+                        a[k] = cmul(a[k], w);
+                        if (b) b[k] = cmul(b[k], w);
+                    }
+                });
+            }
         };
         if constexpr (V >= 2) {
             static_for<0, V / 2>([&](auto h_) {

@@ -12,9 +12,17 @@ static const KernelEntry k_rows[] = {
     B200FFT_ENTRIES_STD(R16384x2), B200FFT_ENTRIES_STD(R16384x4),
 };
 
+static const KernelEntry k_rows_tw[] = {B200FFT_ENTRIES_STD(R4096t15)};
+
 static int default_cluster(int n) { return 1; }
 
 const KernelEntry* find_rows_kernel(int n, bool inverse, int in_dtype, int out_dtype, int cl) {
+    if (cl == 1015) {                                 // test knob: all 15 first-stage twiddle rows from the table
+        const KernelEntry* base = &k_rows_tw[0];
+        for (int i = 0; i < 4; ++i)
+            if (base[i].n == n && base[i].inverse == inverse && base[i].in_dtype == in_dtype && base[i].out_dtype == out_dtype) return &base[i];
+        return nullptr;
+    }
     if (cl == 0) cl = default_cluster(n);
     for (const KernelEntry& e : k_rows)
         if (e.n == n && e.cl == cl && e.inverse == inverse && e.in_dtype == in_dtype && e.out_dtype == out_dtype) return &e;

@@ -258,3 +258,14 @@ def test_config2_full_size(n, batch, dtype):
     """N = 8192 x 16384 and N = 16384 x 8192, Gaussian, seed 2, fp32 and fp16 storage."""
     _sampled_full_size(n, batch, 2, dtype, FWD)
 
+
+
+def test_table_twiddles_variant_matches():
+    """First-stage twiddles all loaded from the table (test knob) against the default,
+    which loads one row and forms the other powers by multiplication."""
+    x = inputs.gaussian_complex64((6, 4096), 96)
+    want = oracle.fft_rows(x.astype(np.complex128), FWD)
+    a = run_fft(to_device_c64(x), 4096, 6, 1, 4096, FWD, C64).cpu().numpy()
+    b = run_fft(to_device_c64(x), 4096, 6, 1, 4096, FWD, C64, options={"cluster": 1015}).cpu().numpy()
+    assert max(worst_rel_l2(a, want)) <= TOL32 and max(worst_rel_l2(b, want)) <= TOL32
+    assert rel_l2(a, b) <= 1e-6
