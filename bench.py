@@ -49,7 +49,9 @@ def measured_peak_gbs():
 
 
 class ClockSampler:
-    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    """Samples the SM clock and the clock-event (throttle) reasons while the timed region
+    runs: NVML from a polling thread every 2 ms, or nvidia-smi every 100 ms if NVML is not
+    importable. Reading only; no setting is changed."""
     FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,"
               "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
               "clocks_event_reasons.sw_power_cap")
@@ -58,8 +60,30 @@ class ClockSampler:
         self.index = index
         self.proc = None
         self.lines = []
+        self.samples = []          # (sm_mhz, reasons bitmask)
+        self.max_mhz = None
+        self.nvml = None
+        self.stop_flag = False
 
     def start(self):
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            idx = self.index
+            vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+            if vis:
+                try:
+                    idx = int(vis.split(",")[self.index])
+                except (ValueError, IndexError):
+                    idx = self.index
+            self.handle = pynvml.nvmlDeviceGetHandleByIndex(idx)
+            self.max_mhz = float(pynvml.nvmlDeviceGetMaxClockInfo(self.handle, pynvml.NVML_CLOCK_SM))
+            self.nvml = pynvml
+            self.thread = threading.Thread(target=self._poll, daemon=True)
+            self.thread.start()
+            return
+        except Exception:
+            self.nvml = None
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}",
@@ -70,13 +94,38 @@ class ClockSampler:
         except Exception:
             self.proc = None
 
+    def _poll(self):
+        n = self.nvml
+        while not self.stop_flag:
+            try:
+                mhz = float(n.nvmlDeviceGetClockInfo(self.handle, n.NVML_CLOCK_SM))
+                try:
+                    rs = int(n.nvmlDeviceGetCurrentClocksEventReasons(self.handle))
+                except Exception:
+                    rs = int(n.nvmlDeviceGetCurrentClocksThrottleReasons(self.handle))
+                self.samples.append((mhz, rs))
+            except Exception:
+                pass
+            time.sleep(0.002)
+
     def _read(self):
         for line in self.proc.stdout:
             self.lines.append(line.strip())
 
     def stop(self):
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        if self.nvml is not None:
+            self.stop_flag = True
+            self.thread.join(timeout=1)
+            n = self.nvml
+            bits = {"hw_slowdown": 0x8, "hw_thermal_slowdown": 0x40, "sw_thermal_slowdown": 0x20, "sw_power_cap": 0x4}
+            reasons = sorted(k for k, b in bits.items() if any(rs & b for _, rs in self.samples))
+            sm = [m for m, _ in self.samples]
+            return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": self.max_mhz,
+                    "sm_min_mhz": float(min(sm)) if sm else None, "reasons": reasons, "samples": len(sm),
+                    "source": "nvml, 2 ms polling during the timed region"}
         if not self.proc:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["clock sampling unavailable"]}
         time.sleep(0.15)
         self.proc.terminate()
         try:
@@ -84,7 +133,6 @@ class ClockSampler:
         except Exception:
             self.proc.kill()
         sm, mx, reasons = [], None, set()
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         for ln in self.lines:
             parts = [p.strip() for p in ln.split(",")]
             if len(parts) < 6:
@@ -98,7 +146,7 @@ class ClockSampler:
                 if val.lower().startswith("active"):
                     reasons.add(nm)
         return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": mx,
-                "reasons": sorted(reasons), "samples": len(sm)}
+                "reasons": sorted(reasons), "samples": len(sm), "source": "nvidia-smi -lms 100"}
 
 
 def dist_env():
@@ -415,6 +463,42 @@ def run_others(torch, B, args, peak):
     return out
 
 
+def run_case(args):
+    """One workload on its own (small JSON line): for profiling a single kernel.
+    --case rows:N:BATCH:c64|c32h[:inverse] | cols:N:BATCH:c64|c32h | sar:c64|c32h"""
+    import torch
+    torch.cuda.set_device(0)
+    from paper_2609_32237_b200 import binding as B
+    peak, _ = measured_peak_gbs()
+    parts = args.case.split(":")
+    kind = parts[0]
+    dt = {"c64": 0, "c32h": 1}
+    stream = torch.cuda.current_stream()
+    if kind in ("rows", "cols"):
+        n, batch, dtype = int(parts[1]), int(parts[2]), dt[parts[3]]
+        direction = 1 if (len(parts) > 4 and parts[4] == "inverse") else -1
+        _, per, _ = bench_fft(torch, B, n, batch, dtype, 2, args.steps, args.warmup, kind, direction)
+        out = summarize(per, metrics.fft_bytes(n, batch, dtype), peak)
+    elif kind == "sar":
+        dtype = dt[parts[1]]
+        sc = inputs.x_band_scene()
+        rd = torch.from_numpy(inputs.simulate_raw(sc, seed=4)).cuda()
+        img = torch.empty_like(rd)
+        p = B.sar_rda_params_create(B.sar_desc_from_scene(sc, dtype))
+        need = B.sar_rda_workspace_bytes(p)
+        ws = torch.empty(need, dtype=torch.uint8, device="cuda")
+        B.sar_rda_set_workspace(p, ws.data_ptr(), need)
+        _, per = time_calls(torch, lambda: B.sar_rda_form_image(rd.data_ptr(), p, img.data_ptr(), stream.cuda_stream),
+                            args.steps, args.warmup, stream)
+        B.sar_rda_params_destroy(p)
+        out = summarize(per, metrics.sar_bytes(4096, 4096, dtype), peak)
+    else:
+        raise SystemExit(f"unknown case {args.case}")
+    out["case"] = args.case
+    print(json.dumps(out))
+    return 0
+
+
 def cpu_baseline(n):
     """The oracle as it stands, timed on this machine's host cores on a bounded sample."""
     import oracle
@@ -432,12 +516,16 @@ def cpu_baseline(n):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--only-main", dest="only_main", action="store_true",
                     help="time only the headline workload (skip the other workloads)")
+    ap.add_argument("--case", default=None,
+                    help="run one workload only, e.g. rows:16384:8192:c64, cols:4096:4096:c64, sar:c64")
     args = ap.parse_args()
+    if args.case:
+        return run_case(args)
     if args.impl == "reference":
         return run_reference(args)
     return run_gpu(args)

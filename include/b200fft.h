@@ -144,7 +144,8 @@ int64_t b200fft_launch_count(void);
  * sinc interpolator; the azimuth filter exp(+j 4 pi R0 (D - 1) / lambda),
  * D = sqrt(1 - (lambda f_a / 2 v)^2); azimuth inverse FFT. Three passes over
  * memory: fused range compression; column FFT; fused RCMC + filter + inverse
- * column FFT.
+ * column FFT (or, by default where the scene allows, RCMC + filter along the
+ * rows followed by the inverse column FFT in place: see sar_rda_set_option).
  * ---------------------------------------------------------------------- */
 typedef struct {
     int64_t n_azimuth;          /* pulses (rows); power of two, 256..16384 */
@@ -170,6 +171,16 @@ int sar_rda_params_create(sar_rda_params_t *params, const sar_rda_desc *desc);
 int sar_rda_workspace_bytes(sar_rda_params_t params, size_t *bytes);
 int sar_rda_set_workspace(sar_rda_params_t params, void *device_ptr, size_t bytes);
 
+/* Variant choice. Key "fused_rcmc": 1 runs step 2 as the single fused kernel
+ * (RCMC + filter + inverse azimuth FFT on column tiles: three passes over
+ * memory in all); 0 runs it as a row pass (RCMC + filter, written to `out`)
+ * followed by the in-place inverse column FFT of `out` (four passes, but
+ * faster on B200; the default whenever the scene allows it). Both give the
+ * same image to rounding. B200FFT_ERR_UNSUPPORTED if the unfused form cannot
+ * serve this scene (migration growing by more than 48 bins over 1024 range
+ * bins, or n_range not a multiple of 1024). */
+int sar_rda_set_option(sar_rda_params_t params, const char *key, int64_t value);
+
 /* raw: DEVICE, n_azimuth x n_range interleaved complex fp32, row-major (row =
  * pulse). out: DEVICE, same shape and type, the focused image; must not alias
  * raw or the workspace. Enqueues three kernels on `stream`; does not
@@ -184,7 +195,7 @@ int sar_rda_form_image_host(const void *host_raw, sar_rda_params_t params, void 
 
 /* Run one step only, for tests: step 0 range compression (raw -> workspace),
  * 1 azimuth FFT (workspace, in place), 2 RCMC + filter + inverse FFT
- * (workspace -> out). `raw` is read by step 0 only, `out` written by step 2 only. */
+ * (workspace -> out; one or two kernels, see sar_rda_set_option). `raw` is read by step 0 only, `out` written by step 2 only. */
 int sar_rda_run_step(const void *raw, sar_rda_params_t params, void *out, int step, void *stream);
 
 int sar_rda_params_destroy(sar_rda_params_t params);

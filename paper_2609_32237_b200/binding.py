@@ -24,7 +24,7 @@ EXPORTS = [
     "fft_execute_host", "fft_plan_destroy", "fft_plan_set_option", "fft_status_string",
     "b200fft_launch_count", "sar_rda_params_create", "sar_rda_workspace_bytes",
     "sar_rda_set_workspace", "sar_rda_form_image", "sar_rda_form_image_host", "sar_rda_run_step",
-    "sar_rda_params_destroy", "fft_execute_noalloc",
+    "sar_rda_params_destroy", "fft_execute_noalloc", "sar_rda_set_option",
 ]
 
 
@@ -69,6 +69,7 @@ def _load():
     L.sar_rda_run_step.argtypes = [vp, vp, vp, ci, vp]
     L.sar_rda_params_destroy.argtypes = [vp]
     L.fft_execute_noalloc.argtypes = [i64, i64, ci, vp, vp, vp]
+    L.sar_rda_set_option.argtypes = [vp, ctypes.c_char_p, i64]
     return L
 
 
@@ -149,6 +150,10 @@ def sar_rda_workspace_bytes(params) -> int:
 
 def sar_rda_set_workspace(params, device_ptr, nbytes):
     _check(_lib.sar_rda_set_workspace(params, device_ptr, nbytes), "sar_rda_set_workspace")
+
+
+def sar_rda_set_option(params, key: str, value: int):
+    _check(_lib.sar_rda_set_option(params, key.encode(), value), "sar_rda_set_option")
 
 
 def sar_rda_form_image(raw_ptr, params, out_ptr, stream=0):

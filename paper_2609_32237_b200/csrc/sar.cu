@@ -14,6 +14,7 @@
 // product exact; a continuous interpolator (evaluated directly, no table);
 // the fractional shift taken from the migration alone.
 #include <cuda_runtime.h>
+#include <cstring>
 #include <new>
 #include "../../include/b200fft.h"
 #include "configs.h"
@@ -290,6 +291,91 @@ __global__ void __launch_bounds__(C::THREADS, 1) sar_rcmc_filter_ifft_kernel(con
     e.template store_last<StoreC64, true>(a.out, (int64_t)n0, a.ld, a.scale);
 }
 
+// ---------------------------------------------------------------- step 2, unfused variant
+// Range cell migration correction and azimuth filter along the rows (range is the
+// contiguous axis, so the 8-tap windows are plain neighbouring samples), written as
+// complex64 into the output image; the inverse azimuth FFT then runs in place on the
+// output with the plain column kernel. One more trip through memory than the fused
+// kernel, but every thread is independent here (no tile-wide barriers), which on this
+// machine is faster than doing the interpolation inside the lock-stepped column tile.
+struct RcmcRows {
+    static constexpr int COLS = 1024;   // range bins per CTA
+    static constexpr int HALO = 64;     // extra staged samples: taps, alignment, growth of the shift over COLS bins
+    static constexpr int TPB = 256;
+};
+
+template <class TIn>
+__global__ void __launch_bounds__(RcmcRows::TPB) sar_rcmc_filter_rows_kernel(const SarArgs a, int chunks) {
+    constexpr int COLS = RcmcRows::COLS, HALO = RcmcRows::HALO, TPB = RcmcRows::TPB;
+    constexpr int EB = TIn::ELEM_BYTES, GRAN = 16 / EB;
+    using elem_t = typename std::conditional<EB == 8, float2, __half2>::type;
+    __shared__ __align__(16) elem_t srow[COLS + HALO];
+    const int k = blockIdx.x / chunks;                 // Doppler bin
+    const int c0 = (blockIdx.x % chunks) * COLS;       // first range bin of this CTA
+    const float4 mg = __ldg(a.tab.mig + k);
+    const float4 ph = __ldg(a.tab.phs + k);
+    const float2 step = __ldg(a.tab.stp + k);
+    int i0;
+    float mu0;
+    migration(mg, c0, i0, mu0);
+    const int start = (c0 + i0 - 3) & ~(GRAN - 1);     // staged window starts on a 16-byte boundary
+    const elem_t* in = reinterpret_cast<const elem_t*>(a.in) + (int64_t)k * a.ld;
+    for (int i = threadIdx.x; i < (COLS + HALO) / GRAN; i += TPB) {
+        const int col = start + i * GRAN;
+        uint4 v = make_uint4(0u, 0u, 0u, 0u);
+        if (col >= 0 && col + GRAN <= a.nr) v = *reinterpret_cast<const uint4*>(in + col);
+        *reinterpret_cast<uint4*>(srow + i * GRAN) = v;
+    }
+    __syncthreads();
+    float2* out = reinterpret_cast<float2*>(a.out) + (int64_t)k * a.ld;
+    const float g = mg.x + mg.y;
+#pragma unroll
+    for (int h = 0; h < COLS / (2 * TPB); ++h) {
+        const int n = c0 + h * 2 * TPB + 2 * threadIdx.x;          // range bins n, n + 1
+        int ia, ib;
+        float mua, mub;
+        migration(mg, n, ia, mua);
+        mub = mua + g;
+        ib = ia;
+        if (mub >= 1.0f) {
+            mub -= 1.0f;
+            ib += 1;
+        }
+        float wa[8], wb[8];
+        sinc8_weights_rcp(mua, wa);
+        sinc8_weights_rcp(mub, wb);
+        const int oa = min(max(n + ia - 3 - start, 0), COLS + HALO - 8);
+        const int ob = min(max(n + 1 + ib - 3 - start, 0), COLS + HALO - 8);
+        float2 sa = make_float2(0.f, 0.f), sb = make_float2(0.f, 0.f);
+#pragma unroll
+        for (int tap = 0; tap < 8; ++tap) {
+            float2 u, w2;
+            if constexpr (EB == 8) {
+                u = srow[oa + tap];
+                w2 = srow[ob + tap];
+            } else {
+                u = __half22float2(srow[oa + tap]);
+                w2 = __half22float2(srow[ob + tap]);
+            }
+            if ((tap - 3) & 1) {
+                sa.x = fmaf(-wa[tap], u.x, sa.x);
+                sa.y = fmaf(-wa[tap], u.y, sa.y);
+                sb.x = fmaf(-wb[tap], w2.x, sb.x);
+                sb.y = fmaf(-wb[tap], w2.y, sb.y);
+            } else {
+                sa.x = fmaf(wa[tap], u.x, sa.x);
+                sa.y = fmaf(wa[tap], u.y, sa.y);
+                sb.x = fmaf(wb[tap], w2.x, sb.x);
+                sb.y = fmaf(wb[tap], w2.y, sb.y);
+            }
+        }
+        const float2 fa = filter_phase(ph, n);
+        const float2 fb = cmul(fa, step);
+        const float2 ya = cmul(sa, fa), yb = cmul(sb, fb);
+        *reinterpret_cast<float4*>(out + n) = make_float4(ya.x, ya.y, yb.x, yb.y);
+    }
+}
+
 // ---------------------------------------------------------------- tables (float64, built once)
 // H[k] = conj( sum_i h[i] exp(-2 pi i k i / nr) ) / nr,  h[i] = exp(j pi K (i/fs)^2), i = -P/2 .. P-P/2-1
 __global__ void sar_build_matched_filter(float2* H, int nr, int pulse_samples, double kappa) {
@@ -394,6 +480,9 @@ struct b200fft_sar_s {
     const SarEntry* range;
     const KernelEntry* azfft;
     const SarEntry* rcmc;
+    const KernelEntry* azifft;   // in-place inverse column transform of the unfused variant
+    bool fused;                  // step 2 as one kernel (true) or as row pass + column pass (false)
+    bool can_unfuse;
     float2 *tw_range, *tw_az, *H;
     float4 *mig, *phs;
     float2* stp;
@@ -434,6 +523,14 @@ extern "C" int sar_rda_params_create(sar_rda_params_t* params, const sar_rda_des
     p->range = find(k_range, nr, dt);
     p->azfft = find_cols_kernel(na, false, dt, dt);
     p->rcmc = find(k_rcmc, na, dt);
+    p->azifft = find_cols_kernel(na, true, B200FFT_C64, B200FFT_C64);
+    {   // the row pass stages COLS + HALO samples: the shift may grow by at most HALO - 16 bins over COLS bins
+        const double aa = wavelength * d->prf_hz / (4.0 * d->velocity_mps), u = aa * aa, sq = sqrt(1.0 - u);
+        const double gmax = u / ((1.0 + sq) * sq);
+        p->can_unfuse = p->azifft != nullptr && nr % RcmcRows::COLS == 0 &&
+                        gmax * RcmcRows::COLS + 16.0 <= (double)RcmcRows::HALO;
+        p->fused = !p->can_unfuse;
+    }
     if (!p->range || !p->azfft || !p->rcmc || d->n_azimuth > 16384 || d->n_range > 16384 || nr % p->rcmc->w) {
         delete p;
         return B200FFT_ERR_UNSUPPORTED;
@@ -512,7 +609,30 @@ extern "C" int sar_rda_run_step(const void* raw, sar_rda_params_t p, void* out, 
     a.in = p->workspace; a.out = out; a.tw = p->tw_az;
     a.tab = SarTables{p->H, p->mig, p->phs, p->stp};
     a.tiles = nr / p->rcmc->w; a.ld = nr; a.nr = (int)nr; a.scale = 1.0f;
-    return p->rcmc->launch(a, st) == cudaSuccess ? B200FFT_OK : B200FFT_ERR_CUDA;
+    if (p->fused) return p->rcmc->launch(a, st) == cudaSuccess ? B200FFT_OK : B200FFT_ERR_CUDA;
+    const int chunks = (int)(nr / RcmcRows::COLS);
+    if (p->d.intermediate_dtype == B200FFT_C64)
+        sar_rcmc_filter_rows_kernel<StoreC64><<<(unsigned)(na * chunks), RcmcRows::TPB, 0, st>>>(a, chunks);
+    else
+        sar_rcmc_filter_rows_kernel<StoreC32H><<<(unsigned)(na * chunks), RcmcRows::TPB, 0, st>>>(a, chunks);
+    g_launch_count.fetch_add(1, std::memory_order_relaxed);
+    if (cudaGetLastError() != cudaSuccess) return B200FFT_ERR_CUDA;
+    FftArgs f{};
+    f.in = out; f.out = out; f.tw = p->tw_az;
+    f.tiles = nr / p->azifft->w; f.dist = nr;
+    f.scale = 1.0f;                         // 1/n_azimuth was applied after the forward azimuth FFT
+    f.prefetch_ahead = 0;
+    return p->azifft->launch(f, st) == cudaSuccess ? B200FFT_OK : B200FFT_ERR_CUDA;
+}
+
+extern "C" int sar_rda_set_option(sar_rda_params_t p, const char* key, int64_t value) {
+    if (!p || !key) return B200FFT_ERR_INVALID_ARG;
+    if (std::strcmp(key, "fused_rcmc") == 0) {
+        if (!value && !p->can_unfuse) return B200FFT_ERR_UNSUPPORTED;
+        p->fused = value != 0;
+        return B200FFT_OK;
+    }
+    return B200FFT_ERR_INVALID_ARG;
 }
 
 extern "C" int sar_rda_form_image(const void* raw, sar_rda_params_t p, void* out, void* stream) {

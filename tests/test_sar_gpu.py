@@ -19,11 +19,13 @@ def _need_gpu():
         pytest.skip("no CUDA device")
 
 
-def _gpu_chain(scene, raw, dtype, steps=False):
+def _gpu_chain(scene, raw, dtype, steps=False, fused=None):
     import torch
     from paper_2609_32237_b200 import binding as B
     p = B.sar_rda_params_create(B.sar_desc_from_scene(scene, dtype))
     try:
+        if fused is not None:
+            B.sar_rda_set_option(p, "fused_rcmc", int(fused))
         need = B.sar_rda_workspace_bytes(p)
         assert need == scene.n_azimuth * scene.n_range * (8 if dtype == C64 else 4)
         ws = torch.zeros(need, dtype=torch.uint8, device="cuda")
@@ -87,6 +89,20 @@ def test_small_scene_fp16_intermediates(small_scene):
         assert quality.peak_cell(got, tuple(cell)) == tuple(cell)
 
 
+@pytest.mark.parametrize("dtype,tol", [(C64, 1e-5), (C32H, 5e-3)])
+def test_small_scene_fused_and_unfused_step2_agree(small_scene, dtype, tol):
+    """Step 2 as one fused kernel and as row pass + in-place column pass: both within
+    tolerance of the oracle, and equal to each other to rounding."""
+    sc, raw, rc, S, img = small_scene
+    a = _gpu_chain(sc, raw, dtype, fused=True)
+    b = _gpu_chain(sc, raw, dtype, fused=False)
+    assert rel_l2(a, img) <= tol and rel_l2(b, img) <= tol
+    assert rel_l2(a, b) <= 2e-6
+    for cell in sc.targets:
+        assert quality.peak_cell(a, tuple(cell)) == tuple(cell)
+        assert quality.peak_cell(b, tuple(cell)) == tuple(cell)
+
+
 def test_single_on_grid_echo_compresses_to_the_pulse_length():
     sc = inputs.x_band_scene(n_azimuth=1024, n_range=2048, n_targets=0)
     sc.noise_variance = 0.0
@@ -99,11 +115,13 @@ def test_single_on_grid_echo_compresses_to_the_pulse_length():
     assert np.abs(inter[0][6]).max() == 0
 
 
+@pytest.mark.parametrize("fused", [False, True])
 @pytest.mark.parametrize("dtype,tol", [(C64, 1e-5), (C32H, 5e-3)])
-def test_config4_full_scene(dtype, tol, full_scene):
-    """4096 x 4096, 16 seeded unit targets, noise at 20 dB: whole image and peak cells."""
+def test_config4_full_scene(dtype, tol, fused, full_scene):
+    """4096 x 4096, 16 seeded unit targets, noise at 20 dB: whole image and peak cells,
+    for both forms of step 2."""
     sc, raw, img = full_scene
-    got = _gpu_chain(sc, raw, dtype)
+    got = _gpu_chain(sc, raw, dtype, fused=fused)
     err = rel_l2(got, img)
     assert err <= tol, err
     for cell in sc.targets:
