@@ -31,7 +31,7 @@ import numpy as np
 ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
-from paper_2609_32237_b200 import inputs, metrics  # noqa: E402
+from paper_2609_32237_b200 import inputs, metrics, multi  # noqa: E402
 
 MAIN = dict(n=4096, batch=32768, seed=1, dtype=0)
 WORKLOAD = "N=4096 batch=32768 complex64 forward, contiguous rows (1 GiB in + 1 GiB out)"
@@ -285,7 +285,7 @@ def run_gpu(args):
     nbytes = metrics.fft_bytes(n, batch, dtype)
 
     # ---- main workload: inputs resident in HBM ---------------------------------
-    x = inputs.gaussian_complex64((batch, n), MAIN["seed"] + rank)
+    x = inputs.gaussian_complex64((batch, n), multi.rank_seed(MAIN["seed"], rank))
     h_in = torch.from_numpy(x).pin_memory()
     h_out = torch.empty_like(h_in).pin_memory()
     d_in = h_in.cuda()
@@ -314,14 +314,11 @@ def run_gpu(args):
     total_ms = e0.elapsed_time(e1)
     launches = B.launch_count() - launches0
     if world > 1:
-        t = torch.tensor([total_ms], device="cuda", dtype=torch.float64)
         dist.barrier()
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
     clocks = sampler.stop() if rank == 0 else None
-    ms_per_step = total_ms / args.steps
-    value = world * nbytes / (ms_per_step * 1e-3) / 1e9
-    kernel_gbs = nbytes / (ms_per_step * 1e-3) / 1e9     # one launch per step: launch duration = step time
+    local_ms_per_step = total_ms / args.steps
+    value, ms_per_step = multi.aggregate_throughput(nbytes, local_ms_per_step, world, device="cuda")
+    kernel_gbs = nbytes / (local_ms_per_step * 1e-3) / 1e9   # one launch per step: launch duration = step time
 
     # ---- end to end: host buffers, copies inside the timed region ------------------
     def step_host():
@@ -339,11 +336,7 @@ def run_gpu(args):
     e1.record(stream)
     torch.cuda.synchronize()
     e2e_ms = e0.elapsed_time(e1)
-    if world > 1:
-        t = torch.tensor([e2e_ms], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item())
-    e2e_value = world * nbytes / (e2e_ms / e2e_steps * 1e-3) / 1e9
+    e2e_value, _ = multi.aggregate_throughput(nbytes, e2e_ms / e2e_steps, world, device="cuda")
     checksum = float(h_out.view(torch.float32)[:8].abs().sum())
     B.fft_plan_destroy(plan)
     del d_in, d_out, h_in, h_out, x
