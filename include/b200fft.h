@@ -102,7 +102,10 @@ int fft_plan_destroy(fft_plan_t plan);
  * share a tile through distributed shared memory; B200FFT_ERR_UNSUPPORTED if
  * that variant is not compiled for the plan's size. Key "prefetch" value d
  * makes each CTA of a rows plan ask L2 for the input of the transform d tiles
- * ahead (0 = off, -1 = the default: one wave ahead for n = 16384). Unknown keys return
+ * ahead (0 = off, -1 = the default: one wave ahead for n = 16384). Key "tma"
+ * value 1 makes a complex64 columns plan (n = 1024, 2048, 4096) stage its tiles
+ * through the tensor memory accelerator (2-D tiled bulk copies, no multicast)
+ * instead of plain vector loads and stores; same results. Unknown keys return
  * B200FFT_ERR_INVALID_ARG. Must be called before set_workspace. */
 int fft_plan_set_option(fft_plan_t plan, const char *key, int64_t value);
 
@@ -135,6 +138,12 @@ const char *fft_status_string(int status);
 /* Number of kernel launches the library has enqueued since it was loaded
  * (all plans, all streams); for launch accounting in benchmarks. */
 int64_t b200fft_launch_count(void);
+
+/* Number of mbarrier waits in the TMA column variant that gave up after their
+ * poll limit since the library was loaded (synchronises the device; 0 unless
+ * something is badly wrong: the waits are bounded so that a lost copy can never
+ * hang the GPU). */
+int b200fft_tma_timeouts(void);
 
 /* ------------------------------------------------------------------------
  * Range-Doppler SAR image formation (paper, Section "End to End:

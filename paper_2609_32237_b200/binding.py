@@ -24,7 +24,7 @@ EXPORTS = [
     "fft_execute_host", "fft_plan_destroy", "fft_plan_set_option", "fft_status_string",
     "b200fft_launch_count", "sar_rda_params_create", "sar_rda_workspace_bytes",
     "sar_rda_set_workspace", "sar_rda_form_image", "sar_rda_form_image_host", "sar_rda_run_step",
-    "sar_rda_params_destroy", "fft_execute_noalloc", "sar_rda_set_option",
+    "sar_rda_params_destroy", "fft_execute_noalloc", "sar_rda_set_option", "b200fft_tma_timeouts",
 ]
 
 
@@ -87,6 +87,10 @@ def _check(status: int, where: str):
 
 def status_string(status: int) -> str:
     return _lib.fft_status_string(status).decode()
+
+
+def tma_timeouts() -> int:
+    return int(_lib.b200fft_tma_timeouts())
 
 
 def launch_count() -> int:

@@ -132,6 +132,17 @@ extern "C" int fft_plan_set_option(fft_plan_t p, const char* key, int64_t value)
         p->prefetch_ahead = (int)value;
         return B200FFT_OK;
     }
+    if (std::strcmp(key, "tma") == 0) {
+        if (p->four_step || p->layout != LAYOUT_COLS || p->dtype != B200FFT_C64) return B200FFT_ERR_UNSUPPORTED;
+        const int old = p->cluster;
+        p->cluster = value ? 77 : 0;
+        int rc = build_single_pass(p);
+        if (rc != B200FFT_OK) {
+            p->cluster = old;
+            return rc;
+        }
+        return B200FFT_OK;
+    }
     if (std::strcmp(key, "cluster") == 0) {
         if (p->four_step || p->n > 16384) return B200FFT_ERR_UNSUPPORTED;
         const int old = p->cluster;
@@ -232,3 +243,5 @@ extern "C" const char* fft_status_string(int status) {
 }
 
 extern "C" int64_t b200fft_launch_count(void) { return g_launch_count.load(); }
+
+extern "C" int b200fft_tma_timeouts(void) { return tma_timeouts(); }

@@ -86,5 +86,6 @@ constexpr KernelEntry make_entry() {
 // cl: CTAs per tile (cluster size); 0 picks the default variant for that size
 const KernelEntry* find_rows_kernel(int n, bool inverse, int in_dtype, int out_dtype, int cl = 0);
 const KernelEntry* find_cols_kernel(int n, bool inverse, int in_dtype, int out_dtype, int cl = 0);
+int tma_timeouts();   // mbarrier waits of the TMA column variant that ran out of polls since load
 
 }  // namespace b200fft
