@@ -85,9 +85,13 @@ int fft_execute(fft_plan_t plan, const void *in, void *out, void *stream);
 
 /* The same transform from HOST buffers (paper's footprint: input plus output):
  * copies host_in -> dev_in, executes dev_in -> dev_out, copies dev_out ->
- * host_out, all enqueued on `stream`. The host buffers should be pinned for
- * the copies to be asynchronous; the device staging buffers are caller-owned
- * and sized like in/out above. Does not synchronise. */
+ * host_out. The host buffers should be pinned for the copies to be
+ * asynchronous; the device staging buffers are caller-owned and sized like
+ * in/out above. Large row batches are cut into 16 chunks whose copy in,
+ * transform and copy out overlap on two internal copy streams (created on the
+ * first such call); towards the caller it is still one operation ordered on
+ * `stream`: it starts after the work already on `stream`, and `stream` waits
+ * for the last copy out. Does not synchronise the host. */
 int fft_execute_host(fft_plan_t plan, const void *host_in, void *host_out,
                      void *dev_in, void *dev_out, void *stream);
 

@@ -28,7 +28,14 @@ struct b200fft_plan_s {
     FourStep fs;                 // two-pass variant
     void* workspace;
     size_t workspace_bytes;
+    // host-buffer path: two copy streams and per-chunk events, created on first use
+    static constexpr int kChunks = 16;
+    cudaStream_t s_in, s_out;
+    cudaEvent_t ev_start, ev_done, ev_in[kChunks], ev_k[kChunks];
+    bool pipe_ready;
 };
+
+static int launch_single_pass(b200fft_plan_s* p, const void* in, void* out, int64_t tiles, cudaStream_t st);
 
 static bool is_pow2(int64_t v) { return v > 0 && (v & (v - 1)) == 0; }
 
@@ -60,6 +67,30 @@ static void release(b200fft_plan_s* p) {
     if (p->tw) cudaFree(p->tw);
     p->tw = nullptr;
     fourstep_release(&p->fs);
+    if (p->pipe_ready) {
+        cudaStreamDestroy(p->s_in);
+        cudaStreamDestroy(p->s_out);
+        cudaEventDestroy(p->ev_start);
+        cudaEventDestroy(p->ev_done);
+        for (int i = 0; i < b200fft_plan_s::kChunks; ++i) {
+            cudaEventDestroy(p->ev_in[i]);
+            cudaEventDestroy(p->ev_k[i]);
+        }
+        p->pipe_ready = false;
+    }
+}
+
+static bool pipe_setup(b200fft_plan_s* p) {
+    if (p->pipe_ready) return true;
+    bool ok = cudaStreamCreateWithFlags(&p->s_in, cudaStreamNonBlocking) == cudaSuccess &&
+              cudaStreamCreateWithFlags(&p->s_out, cudaStreamNonBlocking) == cudaSuccess &&
+              cudaEventCreateWithFlags(&p->ev_start, cudaEventDisableTiming) == cudaSuccess &&
+              cudaEventCreateWithFlags(&p->ev_done, cudaEventDisableTiming) == cudaSuccess;
+    for (int i = 0; ok && i < b200fft_plan_s::kChunks; ++i)
+        ok = cudaEventCreateWithFlags(&p->ev_in[i], cudaEventDisableTiming) == cudaSuccess &&
+             cudaEventCreateWithFlags(&p->ev_k[i], cudaEventDisableTiming) == cudaSuccess;
+    p->pipe_ready = ok;
+    return ok;
 }
 
 extern "C" int fft_plan_create(fft_plan_t* plan, int64_t n, int64_t batch, int64_t stride,
@@ -186,6 +217,11 @@ extern "C" int fft_execute(fft_plan_t p, const void* in, void* out, void* stream
         if (!p->workspace || p->workspace_bytes < need) return B200FFT_ERR_WORKSPACE;
         return fourstep_execute(&p->fs, in, out, p->workspace, st);
     }
+    return launch_single_pass(p, in, out, p->layout == LAYOUT_ROWS ? p->batch : p->batch / p->kernel->w, st);
+}
+
+// one launch of the plan's single-pass kernel over `tiles` tiles starting at in/out
+static int launch_single_pass(b200fft_plan_s* p, const void* in, void* out, int64_t tiles, cudaStream_t st) {
     FftArgs a;
     a.in = in;
     a.out = out;
@@ -199,13 +235,8 @@ extern "C" int fft_execute(fft_plan_t p, const void* in, void* out, void* stream
         a.prefetch_ahead = (p->prefetch_ahead >= 0) ? p->prefetch_ahead : (fills_sm ? p->sms : 0);
     }
     a.scale = (p->direction == B200FFT_INVERSE) ? (float)(1.0 / (double)p->n) : 1.0f;
-    if (p->layout == LAYOUT_ROWS) {
-        a.tiles = p->batch;
-        a.dist = p->dist;
-    } else {
-        a.tiles = p->batch / p->kernel->w;
-        a.dist = p->stride;
-    }
+    a.tiles = tiles;
+    a.dist = (p->layout == LAYOUT_ROWS) ? p->dist : p->stride;
     return p->kernel->launch(a, st) == cudaSuccess ? B200FFT_OK : B200FFT_ERR_CUDA;
 }
 
@@ -215,6 +246,36 @@ extern "C" int fft_execute_host(fft_plan_t p, const void* host_in, void* host_ou
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
     const size_t elems = (size_t)((p->batch - 1) * p->dist + (p->n - 1) * p->stride + 1);
     const size_t bytes = elems * (size_t)elem_bytes(p->dtype);
+    const int CH = b200fft_plan_s::kChunks;
+    if (p->layout == LAYOUT_ROWS && !p->four_step && p->batch >= 4 * CH && bytes >= ((size_t)32 << 20) && pipe_setup(p)) {
+        // Large row batches: cut the batch into chunks and overlap the copy in of chunk i+1,
+        // the transform of chunk i and the copy out of chunk i-1 (PCIe is full duplex). The
+        // caller's stream sees one ordered operation: the copy streams start after everything
+        // already on `st`, and `st` ends up waiting for the last copy out.
+        if (reinterpret_cast<uintptr_t>(dev_in) % 16 || reinterpret_cast<uintptr_t>(dev_out) % 16) return B200FFT_ERR_ALIGNMENT;
+        const size_t eb = (size_t)elem_bytes(p->dtype);
+        bool ok = cudaEventRecord(p->ev_start, st) == cudaSuccess &&
+                  cudaStreamWaitEvent(p->s_in, p->ev_start, 0) == cudaSuccess &&
+                  cudaStreamWaitEvent(p->s_out, p->ev_start, 0) == cudaSuccess;
+        for (int i = 0; ok && i < CH; ++i) {
+            const int64_t b0 = p->batch * i / CH, b1 = p->batch * (i + 1) / CH;
+            const size_t off = (size_t)b0 * (size_t)p->dist * eb;
+            const size_t len = (i + 1 < CH) ? (size_t)(b1 - b0) * (size_t)p->dist * eb : bytes - off;
+            const char* hin = static_cast<const char*>(host_in) + off;
+            char* hout = static_cast<char*>(host_out) + off;
+            char* din = static_cast<char*>(dev_in) + off;
+            char* dout = static_cast<char*>(dev_out) + off;
+            ok = cudaMemcpyAsync(din, hin, len, cudaMemcpyHostToDevice, p->s_in) == cudaSuccess &&
+                 cudaEventRecord(p->ev_in[i], p->s_in) == cudaSuccess &&
+                 cudaStreamWaitEvent(st, p->ev_in[i], 0) == cudaSuccess &&
+                 launch_single_pass(p, din, dout, b1 - b0, st) == B200FFT_OK &&
+                 cudaEventRecord(p->ev_k[i], st) == cudaSuccess &&
+                 cudaStreamWaitEvent(p->s_out, p->ev_k[i], 0) == cudaSuccess &&
+                 cudaMemcpyAsync(hout, dout, len, cudaMemcpyDeviceToHost, p->s_out) == cudaSuccess;
+        }
+        ok = ok && cudaEventRecord(p->ev_done, p->s_out) == cudaSuccess && cudaStreamWaitEvent(st, p->ev_done, 0) == cudaSuccess;
+        return ok ? B200FFT_OK : B200FFT_ERR_CUDA;
+    }
     if (cudaMemcpyAsync(dev_in, host_in, bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return B200FFT_ERR_CUDA;
     int rc = fft_execute(p, dev_in, dev_out, stream);
     if (rc != B200FFT_OK) return rc;
