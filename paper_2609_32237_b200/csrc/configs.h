@@ -31,6 +31,12 @@ using T1024 = Cfg<1024, 4, 32, 1, 1, 16, 4, 16>;
 using T2048 = Cfg<2048, 4, 32, 1, 1, 16, 8, 16>;
 using T4096 = Cfg<4096, 4, 32, 1, 1, 16, 16, 16>;
 using T8192 = Cfg<8192, 2, 32, 1, 1, 16, 32, 16>;
+// wide tiles for the first pass of the two-pass split: whole 128-byte (or 64-byte) row segments
+using F64 = Cfg<64, 16, 32, 4, 1, 16, 4>;
+using F128 = Cfg<128, 16, 32, 2, 1, 16, 8>;
+using F256 = Cfg<256, 16, 32, 1, 1, 16, 16>;
+using F512 = Cfg<512, 16, 32, 1, 1, 16, 2, 16>;
+using F1024 = Cfg<1024, 8, 32, 1, 1, 16, 4, 16>;
 using T2048x2 = Cfg<2048, 4, 32, 1, 2, 16, 8, 16>;
 using T4096x2 = Cfg<4096, 4, 32, 1, 2, 16, 16, 16>;
 using T4096x4 = Cfg<4096, 4, 32, 1, 4, 16, 16, 16>;

@@ -65,9 +65,9 @@ __global__ void __launch_bounds__(C::THREADS, C::MINB) fourstep_pass1_kernel(con
         static_for<0, r>([&](auto j_) {
             constexpr int j = decltype(j_)::value;
             const int64_t k1 = j * KS + b0;
-            const int64_t m0 = (k1 * j2) & nmask, m1 = (m0 + k1) & nmask;
+            const int64_t m0 = (k1 * j2) & nmask;
             const float2 w0 = cmul(__ldg(a.tw_hi + (m0 >> 10)), __ldg(a.tw_lo + (m0 & 1023)));
-            const float2 w1 = cmul(__ldg(a.tw_hi + (m1 >> 10)), __ldg(a.tw_lo + (m1 & 1023)));
+            const float2 w1 = cmul(w0, __ldg(a.tw_lo + k1));     // one column on: times exp(-2 pi i k1 / n), k1 < 1024
             TOut::store2(a.out, b * a.dist_out + k1 * a.n2 + j2, cmul(e.x[j * V + v], w0), cmul(e.x[j * V + v + 1], w1));
         });
     });
@@ -123,8 +123,8 @@ constexpr FourStepEntry make_fs_entry() {
     make_fs_entry<C, false, StoreC64, PASS>(), make_fs_entry<C, true, StoreC64, PASS>(), \
     make_fs_entry<C, false, StoreC32H, PASS>(), make_fs_entry<C, true, StoreC32H, PASS>()
 
-static const FourStepEntry k_pass1[] = {FS_ENTRIES(T64, 1), FS_ENTRIES(T128, 1), FS_ENTRIES(T256, 1),
-                                        FS_ENTRIES(T512, 1), FS_ENTRIES(T1024, 1)};
+static const FourStepEntry k_pass1[] = {FS_ENTRIES(F64, 1), FS_ENTRIES(F128, 1), FS_ENTRIES(F256, 1),
+                                        FS_ENTRIES(F512, 1), FS_ENTRIES(F1024, 1)};
 static const FourStepEntry k_pass2[] = {FS_ENTRIES(T64, 2), FS_ENTRIES(T128, 2), FS_ENTRIES(T256, 2),
                                         FS_ENTRIES(T512, 2), FS_ENTRIES(T1024, 2)};
 
