@@ -44,7 +44,7 @@ static int elem_bytes(int dtype) { return dtype == B200FFT_C64 ? 8 : 4; }
 static int build_single_pass(b200fft_plan_s* p) {
     const bool inv = p->direction == B200FFT_INVERSE;
     const KernelEntry* k = (p->layout == LAYOUT_ROWS)
-                               ? find_rows_kernel((int)p->n, inv, p->dtype, p->dtype, p->cluster)
+                               ? find_rows_kernel((int)p->n, inv, p->dtype, p->dtype, p->cluster, p->batch)
                                : find_cols_kernel((int)p->n, inv, p->dtype, p->dtype, p->cluster);
     if (!k) return B200FFT_ERR_UNSUPPORTED;
     if (p->kernel && p->kernel->tw_total == k->tw_total) {   // same factorisation: the table is reusable

@@ -84,7 +84,8 @@ constexpr KernelEntry make_entry() {
     make_entry<C, true, StoreC32H, StoreC32H>()
 
 // cl: CTAs per tile (cluster size); 0 picks the default variant for that size
-const KernelEntry* find_rows_kernel(int n, bool inverse, int in_dtype, int out_dtype, int cl = 0);
+const KernelEntry* find_rows_kernel(int n, bool inverse, int in_dtype, int out_dtype, int cl = 0,
+                                    int64_t batch = (int64_t)1 << 40);
 const KernelEntry* find_cols_kernel(int n, bool inverse, int in_dtype, int out_dtype, int cl = 0);
 int tma_timeouts();   // mbarrier waits of the TMA column variant that ran out of polls since load
 

@@ -308,3 +308,11 @@ def test_execute_host_pipelined_and_simple_paths():
         idx = inputs.sample_indices(batch, 8, 3)
         want = oracle.fft_rows(x[idx].astype(np.complex128))
         assert max(worst_rel_l2(h_out.numpy()[idx], want)) <= TOL32
+
+
+def test_small_batches_pick_the_split_transform_variant():
+    """Batches too small to fill the SMs default to a transform split over a cluster of
+    CTAs (N = 16384: batch <= 32; N = 8192: batch <= 16): parity at the switch-over sizes."""
+    for n, batch in ((16384, 32), (16384, 33), (8192, 16), (8192, 17), (16384, 2)):
+        _check_rows(n, batch, seed=98, gaussian=True)
+        _check_rows(n, batch, seed=99, direction=INV)
