@@ -142,3 +142,52 @@ def full_scene():
     raw = inputs.simulate_raw(sc, seed=4)
     img = oracle.sar_rda(oracle.sar_params(sc), raw)
     return sc, raw, img
+
+
+def test_other_frame_sizes_and_error_paths():
+    """A 2048 x 1024 frame with a 5 us pulse (other kernel instantiations), both intermediate
+    types and both forms of step 2; then the host-side error paths of the SAR calls."""
+    import torch
+    from paper_2609_32237_b200 import binding as B
+    sc = inputs.x_band_scene(n_azimuth=2048, n_range=1024, n_targets=0)
+    sc.antenna_m = 1.5
+    sc.pulse_s = 5e-6
+    sc.targets = inputs.seeded_target_cells(sc, 3, seed=11)
+    raw = inputs.simulate_raw(sc, seed=11)
+    img = oracle.sar_rda(oracle.sar_params(sc), raw)
+    for dtype, tol in ((C64, 1e-5), (C32H, 5e-3)):
+        for fused in (False, True):
+            got = _gpu_chain(sc, raw, dtype, fused=fused)
+            assert rel_l2(got, img) <= tol
+            for cell in sc.targets:
+                assert quality.peak_cell(got, tuple(cell)) == tuple(cell)
+    p = B.sar_rda_params_create(B.sar_desc_from_scene(sc, C64))
+    try:
+        rd = to_device_c64(raw)
+        out = torch.zeros_like(rd)
+        with pytest.raises(B.B200FftError) as e:               # no workspace yet
+            B.sar_rda_form_image(rd.data_ptr(), p, out.data_ptr(), 0)
+        assert e.value.status == 6
+        need = B.sar_rda_workspace_bytes(p)
+        small = torch.zeros(need // 2, dtype=torch.uint8, device="cuda")
+        with pytest.raises(B.B200FftError) as e:
+            B.sar_rda_set_workspace(p, small.data_ptr(), need // 2)
+        assert e.value.status == 6
+        ws = torch.zeros(need, dtype=torch.uint8, device="cuda")
+        B.sar_rda_set_workspace(p, ws.data_ptr(), need)
+        with pytest.raises(B.B200FftError) as e:               # output must not alias the input
+            B.sar_rda_form_image(rd.data_ptr(), p, rd.data_ptr(), 0)
+        assert e.value.status == 1
+        with pytest.raises(B.B200FftError) as e:
+            B.sar_rda_set_option(p, "no_such_option", 1)
+        assert e.value.status == 1
+        with pytest.raises(B.B200FftError) as e:
+            B.sar_rda_run_step(rd.data_ptr(), p, out.data_ptr(), 7, 0)
+        assert e.value.status == 1
+    finally:
+        B.sar_rda_params_destroy(p)
+    bad = B.sar_desc_from_scene(sc, C64)
+    bad.n_azimuth = 512                                          # not a compiled azimuth size
+    with pytest.raises(B.B200FftError) as e:
+        B.sar_rda_params_create(bad)
+    assert e.value.status == 2
