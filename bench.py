@@ -492,6 +492,51 @@ def run_case(args):
     return 0
 
 
+def run_sweep(args):
+    """Hot versus cold throughput of the N=4096 kernel against the batch footprint (the
+    paper's Table "One 4096-Point Kernel vs. Batch Size"): hot = back-to-back launches on
+    the same buffers, cold = a 512 MiB scratch write before every launch."""
+    import torch
+    torch.cuda.set_device(0)
+    from paper_2609_32237_b200 import binding as B
+    peak, _ = measured_peak_gbs()
+    stream = torch.cuda.current_stream()
+    scratch = torch.empty(512 << 20, dtype=torch.uint8, device="cuda")
+    n, rows = 4096, []
+    for batch in (16, 64, 148, 296, 592, 1184, 2048, 4096, 8192, 16384, 32768):
+        x = torch.randn(batch, n, 2, device="cuda")
+        y = torch.empty_like(x)
+        plan = B.fft_plan_create(n, batch, 1, n, -1, 0)
+        call = lambda: B.fft_execute(plan, x.data_ptr(), y.data_ptr(), stream.cuda_stream)
+        reps = max(20, min(2000, (256 << 20) // (batch * n * 16)))
+        for _ in range(5):
+            call()
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        for _ in range(reps):
+            call()
+        b.record(stream)
+        torch.cuda.synchronize()
+        hot_ms = a.elapsed_time(b) / reps
+        cold = []
+        for _ in range(9):
+            scratch.zero_()
+            a.record(stream)
+            call()
+            b.record(stream)
+            torch.cuda.synchronize()
+            cold.append(a.elapsed_time(b))
+        cold_ms = float(np.median(cold))
+        B.fft_plan_destroy(plan)
+        nb = metrics.fft_bytes(n, batch, 0)
+        rows.append({"batch": batch, "footprint_mib": nb / 2 ** 20, "hot_gbs": nb / hot_ms / 1e6,
+                     "cold_gbs": nb / cold_ms / 1e6, "hot_us": hot_ms * 1e3, "cold_us": cold_ms * 1e3,
+                     "hot_gflops": metrics.fft_gflops(n, batch, hot_ms * 1e-3)})
+    print(json.dumps({"sweep": "N=4096 c64 forward, hot vs cold", "hbm_peak_gbs": peak, "rows": rows}))
+    return 0
+
+
 def cpu_baseline(n):
     """The oracle as it stands, timed on this machine's host cores on a bounded sample."""
     import oracle
@@ -516,7 +561,10 @@ def main():
                     help="time only the headline workload (skip the other workloads)")
     ap.add_argument("--case", default=None,
                     help="run one workload only, e.g. rows:16384:8192:c64, cols:4096:4096:c64, sar:c64")
+    ap.add_argument("--sweep", action="store_true", help="hot vs cold throughput against the batch footprint")
     args = ap.parse_args()
+    if args.sweep:
+        return run_sweep(args)
     if args.case:
         return run_case(args)
     if args.impl == "reference":
