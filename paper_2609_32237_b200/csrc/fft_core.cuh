@@ -211,7 +211,7 @@ struct Cfg {
     // registers per thread are capped at 128 so that at least 65536 / (128 * THREADS) CTAs fit an SM
     static constexpr int MINB = (65536 / (128 * THREADS)) > 0 ? (65536 / (128 * THREADS)) : 1;
     static_assert(P_ % R1_ == 0 && P_ % R2_ == 0 && P_ % R3_ == 0 && P_ % R4_ == 0, "P must be a multiple of every radix");
-    static_assert(P_ / R1_ >= 2 && P_ / radix(S) >= 2, "first and last stage need two butterflies per thread for 128-bit access");
+    static_assert(P_ / radix(S) >= 2, "the last stage needs two butterflies per thread (128-bit stores)");
     static_assert((N_ * W_) % (P_ * CL_) == 0, "tile must divide among threads");
 };
 
@@ -448,11 +448,19 @@ struct Engine {
         // ones (w^k = w^M w^(k-M)). Only the first stage of a one-transform tile trades
         // loads for arithmetic: there every lane needs different entries, so each table row
         // costs four L1 wavefronts per warp, and L1 is the busiest unit of these kernels.
-        constexpr int M = (s == 1 && W == 1 && V >= 2 && r > C::TW1_LOADS) ? C::TW1_LOADS : r - 1;
+        constexpr int M = (s == 1 && W == 1 && r > C::TW1_LOADS) ? C::TW1_LOADS : r - 1;
         auto twiddle_pair = [&](int lo0, float2* a, float2* b) {
             // a, b: the r values of butterflies v, v+1 (b == nullptr if V == 1)
             const float2* row = tw + C::tw_off(s) + lo0;
-            if constexpr (M < r - 1) {
+            if constexpr (M < r - 1 && V == 1) {
+                float2 wa[r];
+                static_for<1, r>([&](auto k_) {
+                    constexpr int k = decltype(k_)::value;
+                    if constexpr (k <= M) wa[k] = __ldg(row + (k - 1) * Ls);
+                    else wa[k] = cmul(wa[M], wa[k - M]);
+                    a[k] = cmul(a[k], wa[k]);
+                });
+            } else if constexpr (M < r - 1) {
                 float2 wa[r], wb[r];
                 static_for<1, r>([&](auto k_) {
                     constexpr int k = decltype(k_)::value;
@@ -526,6 +534,17 @@ struct Engine {
     __device__ __forceinline__ void load_first(const void* in, int64_t base, int64_t ld) {
         using G = Geo<C, 1>;
         constexpr int V = G::V, r = G::r;
+        if constexpr (V == 1) {     // radix = values per thread: one butterfly per thread, 64-bit loads,
+                                    // still one contiguous run per warp
+            const int c = C::template cidx<1>(t, 0, rank);
+            const int q = c % W, lo = c / W;
+            static_for<0, r>([&](auto j_) {
+                constexpr int j = decltype(j_)::value;
+                const int64_t idx = (W == 1) ? base + j * G::Ls + lo : base + (int64_t)(j * G::Ls + lo) * ld + q;
+                x[j] = ST::load1(in, idx);
+                if constexpr (CONJ) x[j].y = -x[j].y;
+            });
+        }
         static_for<0, V / 2>([&](auto h_) {
             constexpr int v = 2 * decltype(h_)::value;
             const int c = C::template cidx<V>(t, v, rank);

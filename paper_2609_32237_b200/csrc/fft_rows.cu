@@ -12,7 +12,7 @@ static const KernelEntry k_rows[] = {
     B200FFT_ENTRIES_STD(R16384x2), B200FFT_ENTRIES_STD(R16384x4),
 };
 
-static const KernelEntry k_rows_tw[] = {B200FFT_ENTRIES_STD(R4096t15)};
+static const KernelEntry k_rows_alt[] = {B200FFT_ENTRIES_STD(R4096t15), B200FFT_ENTRIES_STD(R16384s4)};
 
 // Small batches leave most SMs idle with one CTA per transform (the paper's "when not to
 // use it"): there a transform is split over a cluster of CTAs through distributed shared
@@ -25,10 +25,10 @@ static int default_cluster(int n, int64_t batch) {
 }
 
 const KernelEntry* find_rows_kernel(int n, bool inverse, int in_dtype, int out_dtype, int cl, int64_t batch) {
-    if (cl == 1015) {                                 // test knob: all 15 first-stage twiddle rows from the table
-        const KernelEntry* base = &k_rows_tw[0];
-        for (int i = 0; i < 4; ++i)
-            if (base[i].n == n && base[i].inverse == inverse && base[i].in_dtype == in_dtype && base[i].out_dtype == out_dtype) return &base[i];
+    if (cl == 1015 || cl == 1016) {                   // test knobs: 1015 = all first-stage twiddle rows from
+                                                      // the table (n = 4096); 1016 = four-stage n = 16384
+        for (const KernelEntry& e : k_rows_alt)
+            if (e.n == n && e.inverse == inverse && e.in_dtype == in_dtype && e.out_dtype == out_dtype) return &e;
         return nullptr;
     }
     if (cl == 0) cl = default_cluster(n, batch);

@@ -47,11 +47,7 @@ static int build_single_pass(b200fft_plan_s* p) {
                                ? find_rows_kernel((int)p->n, inv, p->dtype, p->dtype, p->cluster, p->batch)
                                : find_cols_kernel((int)p->n, inv, p->dtype, p->dtype, p->cluster);
     if (!k) return B200FFT_ERR_UNSUPPORTED;
-    if (p->kernel && p->kernel->tw_total == k->tw_total) {   // same factorisation: the table is reusable
-        p->kernel = k;
-        return B200FFT_OK;
-    }
-    p->kernel = k;
+    p->kernel = k;                  // the table depends on the factorisation: always rebuilt
     if (p->tw) cudaFree(p->tw);
     p->tw = nullptr;
     if (cudaMalloc(&p->tw, sizeof(float2) * (size_t)p->kernel->tw_total) != cudaSuccess) {

@@ -269,6 +269,12 @@ def test_table_twiddles_variant_matches():
     b = run_fft(to_device_c64(x), 4096, 6, 1, 4096, FWD, C64, options={"cluster": 1015}).cpu().numpy()
     assert max(worst_rel_l2(a, want)) <= TOL32 and max(worst_rel_l2(b, want)) <= TOL32
     assert rel_l2(a, b) <= 1e-6
+    # the four-stage factorisation of 16384 (16 x 4 x 16 x 16) against the default 32 x 32 x 16
+    x = inputs.gaussian_complex64((3, 16384), 94)
+    want = oracle.fft_rows(x.astype(np.complex128), INV)
+    a = run_fft(to_device_c64(x), 16384, 3, 1, 16384, INV, C64).cpu().numpy()
+    b = run_fft(to_device_c64(x), 16384, 3, 1, 16384, INV, C64, options={"cluster": 1016}).cpu().numpy()
+    assert max(worst_rel_l2(a, want)) <= TOL32 and max(worst_rel_l2(b, want)) <= TOL32
 
 
 @pytest.mark.parametrize("n", [1024, 2048, 4096])
