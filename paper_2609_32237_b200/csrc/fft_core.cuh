@@ -588,6 +588,12 @@ struct Engine {
     // ---- global store with the last-stage mapping: X[b0 + (N / r_S) j] ---------------------
     template <class ST, bool CONJ>
     __device__ __forceinline__ void store_last(void* out, int64_t base, int64_t ld, float scale) {
+        // the unnormalised forward transform (scale 1) skips the two multiplications per value
+        if (scale == 1.0f) store_last_impl<ST, CONJ, false>(out, base, ld, scale);
+        else store_last_impl<ST, CONJ, true>(out, base, ld, scale);
+    }
+    template <class ST, bool CONJ, bool SCALE>
+    __device__ __forceinline__ void store_last_impl(void* out, int64_t base, int64_t ld, float scale) {
         using G = Geo<C, S>;
         constexpr int V = G::V, r = G::r;
         constexpr int KS = C::N / r;
@@ -599,8 +605,14 @@ struct Engine {
                 constexpr int j = decltype(j_)::value;
                 const int64_t idx = (W == 1) ? base + j * KS + b0 : base + (int64_t)(j * KS + b0) * ld + q;
                 float2 a = x[j * V + v], b = x[j * V + v + 1];
-                a = make_float2(a.x * scale, (CONJ ? -a.y : a.y) * scale);
-                b = make_float2(b.x * scale, (CONJ ? -b.y : b.y) * scale);
+                if constexpr (CONJ) {
+                    a.y = -a.y;
+                    b.y = -b.y;
+                }
+                if constexpr (SCALE) {
+                    a = make_float2(a.x * scale, a.y * scale);
+                    b = make_float2(b.x * scale, b.y * scale);
+                }
                 ST::store2(out, idx, a, b);
             });
         });
