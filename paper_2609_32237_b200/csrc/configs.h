@@ -16,7 +16,7 @@ using R8192 = Cfg<8192, 1, 32, 1, 1, 16, 32, 16>;
 // 16384 = 32 x 32 x 16: two exchanges instead of three; its radix-32 first stage has one
 // butterfly per thread, so the global loads are 64 bits per thread (still one contiguous
 // run per warp); measured 6-10 % faster than 16 x 4 x 16 x 16, which stays as a test knob
-using R16384 = Cfg<16384, 1, 32, 1, 1, 32, 32, 16>;
+using R16384 = Cfg<16384, 1, 32, 1, 1, 32, 32, 16, 1, 4>;   // 4 of the 31 first-stage twiddle rows loaded
 using R16384s4 = Cfg<16384, 1, 32, 1, 1, 16, 4, 16, 16>;
 // the same transforms split over a cluster of 2 or 4 CTAs (smaller tiles per SM, more CTAs resident)
 using R8192x2 = Cfg<8192, 1, 32, 1, 2, 16, 32, 16>;
@@ -25,6 +25,7 @@ using R16384x2 = Cfg<16384, 1, 32, 1, 2, 16, 4, 16, 16>;
 using R16384x4 = Cfg<16384, 1, 32, 1, 4, 16, 4, 16, 16>;
 // the same with every first-stage twiddle row loaded from the table instead of computed
 using R4096t15 = Cfg<4096, 1, 32, 1, 1, 16, 16, 16, 1, 15>;
+
 
 // W adjacent columns (or rows, in the second pass of the two-pass split) per tile
 using T64 = Cfg<64, 4, 32, 16, 1, 16, 4>;
