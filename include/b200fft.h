@@ -56,8 +56,8 @@ typedef struct b200fft_sar_s *sar_rda_params_t;
  *   columns  dist == 1, stride >= batch, stride and batch even: the columns of
  *            a row-major matrix (paper, Section "End to End": the FFT that
  *            reads the columns directly)
- * Supported sizes: n a power of two, 256 <= n <= 16384 in a single pass over
- * memory; 2^15 <= n <= 2^20 (rows only) by a two-pass four-step split (the
+ * Supported sizes: n a power of two, 32 <= n <= 16384 in a single pass over
+ * memory (columns: 256 <= n <= 8192); 2^15 <= n <= 2^20 (rows only) by a two-pass four-step split (the
  * paper's "usual remedy when a transform does not fit on chip"), which needs a
  * workspace of n*batch elements of the storage type.
  *

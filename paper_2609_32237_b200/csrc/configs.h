@@ -7,6 +7,10 @@
 namespace b200fft {
 
 // contiguous rows, one transform per tile
+// (the three smallest keep 16 values per thread: 8, 4 and 2 threads per transform)
+using R128 = Cfg<128, 1, 16, 16, 1, 16, 8>;
+using R64 = Cfg<64, 1, 16, 32, 1, 8, 8>;
+using R32 = Cfg<32, 1, 16, 64, 1, 4, 8>;
 using R256 = Cfg<256, 1, 32, 16, 1, 16, 16>;
 using R512 = Cfg<512, 1, 32, 8, 1, 16, 2, 16>;
 using R1024 = Cfg<1024, 1, 32, 4, 1, 16, 4, 16>;

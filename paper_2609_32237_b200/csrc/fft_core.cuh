@@ -204,7 +204,9 @@ struct Cfg {
         return w;
     }
     static_assert(R1_ * R2_ * R3_ * R4_ == N_, "radices must multiply to N");
-    static_assert(L(1) * W_ >= 16, "the swizzle permutes 16-element groups below the top digit");
+    // bits of the element index the swizzle may flip: bits 1..3, but only below the top digit
+    static constexpr int SWZ = 14 & (L(1) * W_ - 1);
+    static_assert(L(1) * W_ >= 2, "at least two elements below the top digit");
     static_assert(CL_ == 1 || G_ == 1, "a cluster works on one tile");
     static_assert(CL_ >= 1 && R1_ % CL_ == 0 && RC >= 2, "the cluster splits the top digit");
     static_assert(CL_ == 1 || RC * W_ >= 16 || L(2) * W_ >= 16, "second digit must stay constant over 16 elements");
@@ -274,12 +276,12 @@ struct Geo {
     __device__ __forceinline__ int elem() const {
         if constexpr (s == 1) {
             constexpr int jl = j % RC;                // top digit relative to the owner
-            return (e0 + jl * estep) ^ (((bl0 + jl) * W) & 14);
+            return (e0 + jl * estep) ^ (((bl0 + jl) * W) & C::SWZ);
         } else if constexpr (!last) {
-            if constexpr (C::blw(s) < 16) return (e0 + j * estep) ^ (((bl0 + j * C::blw(s)) * W) & 14);
-            else return (e0 + j * estep) ^ ((bl0 * W) & 14);
+            if constexpr (C::blw(s) < 16) return (e0 + j * estep) ^ (((bl0 + j * C::blw(s)) * W) & C::SWZ);
+            else return (e0 + j * estep) ^ ((bl0 * W) & C::SWZ);
         } else {
-            return (e0 + j * estep) ^ ((bl0 * W) & 14);
+            return (e0 + j * estep) ^ ((bl0 * W) & C::SWZ);
         }
     }
 };

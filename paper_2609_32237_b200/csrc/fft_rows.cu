@@ -5,6 +5,7 @@
 namespace b200fft {
 
 static const KernelEntry k_rows[] = {
+    B200FFT_ENTRIES_STD(R32),   B200FFT_ENTRIES_STD(R64),   B200FFT_ENTRIES_STD(R128),
     B200FFT_ENTRIES_STD(R256),  B200FFT_ENTRIES_STD(R512),
     B200FFT_ENTRIES_STD(R1024), B200FFT_ENTRIES_STD(R2048), B200FFT_ENTRIES_STD(R4096),
     B200FFT_ENTRIES_STD(R8192), B200FFT_ENTRIES_STD(R16384),

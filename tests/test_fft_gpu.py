@@ -362,3 +362,18 @@ def test_seeded_random_plans_against_the_oracle():
                 got = half_to_c128(run_fft(to_device_half(h), n, cols, ld, 1, direction, C32H))[:, :cols]
             worst = pooled = rel_l2(got, want)
         assert worst <= tol and pooled <= tol, (trial, layout, n, dtype, direction, worst)
+
+
+@pytest.mark.parametrize("n", [32, 64, 128])
+def test_small_transforms(n):
+    """N = 32, 64, 128: several transforms per CTA, ragged batches, both directions, padding,
+    fp16 storage; each against the direct DFT."""
+    for batch in (1, 5, 130, 1000):
+        _check_rows(n, batch, seed=300 + n + batch, gaussian=(batch == 130))
+        _check_rows(n, batch, seed=301 + n + batch, direction=INV)
+    _check_rows(n, 37, seed=302, dist=n + 6)
+    x = inputs.gaussian_complex64((77, n), 303)
+    h = inputs.to_half_storage(x)
+    want = oracle.fft_rows(inputs.from_half_storage(h), FWD)
+    got = half_to_c128(run_fft(to_device_half(h), n, 77, 1, n, FWD, C32H))
+    assert max(worst_rel_l2(got, want)) <= TOL16
