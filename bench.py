@@ -215,7 +215,8 @@ def flush_l2(torch, scratch):
     scratch.zero_()
 
 
-def bench_fft(torch, B, n, batch, dtype, seed, steps, warmup, layout="rows", direction=-1, cold_flush=None):
+def bench_fft(torch, B, n, batch, dtype, seed, steps, warmup, layout="rows", direction=-1, cold_flush=None,
+              options=None):
     stream = torch.cuda.current_stream()
     if layout == "rows":
         x = inputs.gaussian_complex64((batch, n), seed)
@@ -223,6 +224,8 @@ def bench_fft(torch, B, n, batch, dtype, seed, steps, warmup, layout="rows", dir
     else:
         x = inputs.uniform_complex64((n, batch), seed)
         plan = B.fft_plan_create(n, batch, batch, 1, direction, dtype)
+    for key, value in (options or {}).items():
+        B.fft_plan_set_option(plan, key, value)
     if dtype == 0:
         d_in = torch.from_numpy(x).cuda()
     else:
@@ -470,7 +473,8 @@ def run_case(args):
     if kind in ("rows", "cols"):
         n, batch, dtype = int(parts[1]), int(parts[2]), dt[parts[3]]
         direction = 1 if (len(parts) > 4 and parts[4] == "inverse") else -1
-        _, per, _ = bench_fft(torch, B, n, batch, dtype, 2, args.steps, args.warmup, kind, direction)
+        options = dict((kv.split("=")[0], int(kv.split("=")[1])) for kv in args.option)
+        _, per, _ = bench_fft(torch, B, n, batch, dtype, 2, args.steps, args.warmup, kind, direction, options=options)
         out = summarize(per, metrics.fft_bytes(n, batch, dtype), peak)
     elif kind == "sar":
         dtype = dt[parts[1]]
@@ -561,6 +565,8 @@ def main():
                     help="time only the headline workload (skip the other workloads)")
     ap.add_argument("--case", default=None,
                     help="run one workload only, e.g. rows:16384:8192:c64, cols:4096:4096:c64, sar:c64")
+    ap.add_argument("--option", action="append", default=[],
+                    help="with --case rows/cols: plan option KEY=VALUE (repeatable), e.g. cluster=4")
     ap.add_argument("--sweep", action="store_true", help="hot vs cold throughput against the batch footprint")
     args = ap.parse_args()
     if args.sweep:

@@ -109,7 +109,14 @@ int fft_plan_destroy(fft_plan_t plan);
  * ahead (0 = off, -1 = the default: one wave ahead for n = 16384). Key "tma"
  * value 1 makes a complex64 columns plan (n = 1024, 2048, 4096) stage its tiles
  * through the tensor memory accelerator (2-D tiled bulk copies, no multicast)
- * instead of plain vector loads and stores; same results. Unknown keys return
+ * instead of plain vector loads and stores; same results. Key "staged" value
+ * 1 makes a rows plan with n = 16384 run as a persistent kernel (one CTA per
+ * multiprocessor looping over transforms) whose next transform arrives in
+ * shared memory through untiled bulk copies while the current one is computed;
+ * 0 forbids it, -1 restores the default (on for fp16 storage with a batch of
+ * at least two transforms per multiprocessor); B200FFT_ERR_UNSUPPORTED for
+ * other sizes; same results. Every wait on such a copy is bounded:
+ * b200fft_tma_timeouts() counts waits that gave up. Unknown keys return
  * B200FFT_ERR_INVALID_ARG. Must be called before set_workspace. */
 int fft_plan_set_option(fft_plan_t plan, const char *key, int64_t value);
 
@@ -143,8 +150,8 @@ const char *fft_status_string(int status);
  * (all plans, all streams); for launch accounting in benchmarks. */
 int64_t b200fft_launch_count(void);
 
-/* Number of mbarrier waits in the TMA column variant that gave up after their
- * poll limit since the library was loaded (synchronises the device; 0 unless
+/* Number of mbarrier waits in the TMA column variant and the staged rows
+ * variant that gave up after their poll limit since the library was loaded (synchronises the device; 0 unless
  * something is badly wrong: the waits are bounded so that a lost copy can never
  * hang the GPU). */
 int b200fft_tma_timeouts(void);

@@ -1,5 +1,6 @@
-// Thin wrappers over the tensor memory accelerator (2-D tiled cp.async.bulk.tensor, no
-// multicast) and mbarrier, as used by the TMA variant of the column-tile kernel.
+// Thin wrappers over the tensor memory accelerator (2-D tiled cp.async.bulk.tensor and untiled
+// cp.async.bulk, no multicast) and mbarrier, as used by the TMA variant of the column-tile
+// kernel and the staged persistent row kernel.
 #pragma once
 #include <cstdint>
 
@@ -35,6 +36,15 @@ __device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.comm
 __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 // make generic-proxy writes to shared memory visible to the asynchronous proxy
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+// Untiled bulk copy global -> shared memory of this CTA, completion counted in bytes on `bar`;
+// both addresses 16-byte aligned, `bytes` a multiple of 16.
+__device__ __forceinline__ void bulk_load_1d(void* smem_dst, const void* gsrc, unsigned bytes, uint64_t* bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                     smem_u32(smem_dst)),
+                 "l"(gsrc), "r"(bytes), "r"(smem_u32(bar))
+                 : "memory");
+}
 
 // 2-D tiled TMA: box {bx, by} of the tensor described by `tmap`, at coordinates (x, y);
 // x times the element size must be a multiple of 16 bytes.

@@ -88,5 +88,6 @@ const KernelEntry* find_rows_kernel(int n, bool inverse, int in_dtype, int out_d
                                     int64_t batch = (int64_t)1 << 40);
 const KernelEntry* find_cols_kernel(int n, bool inverse, int in_dtype, int out_dtype, int cl = 0);
 int tma_timeouts();   // mbarrier waits of the TMA column variant that ran out of polls since load
+int rows_stage_timeouts();   // the same for the staged persistent row kernels
 
 }  // namespace b200fft

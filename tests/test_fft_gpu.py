@@ -377,3 +377,53 @@ def test_small_transforms(n):
     want = oracle.fft_rows(inputs.from_half_storage(h), FWD)
     got = half_to_c128(run_fft(to_device_half(h), n, 77, 1, n, FWD, C32H))
     assert max(worst_rel_l2(got, want)) <= TOL16
+
+
+@pytest.mark.parametrize("n,batch", [(16384, 5), (16384, 300), (16384, 449)])
+@pytest.mark.parametrize("dtype", [C64, C32H])
+def test_staged_persistent_rows(n, batch, dtype):
+    """The persistent row kernel whose next tile arrives through the copy engine while the
+    current one is transformed: fewer tiles than CTAs, several tiles per CTA with a ragged
+    last round, both directions and storage types; no bounded wait ran out."""
+    from paper_2609_32237_b200 import binding as B
+    x = inputs.gaussian_complex64((batch, n), 300 + batch)
+    rows = inputs.sample_indices(batch, 6, seed=batch)
+    for direction in (FWD, INV):
+        if dtype == C64:
+            got = run_fft(to_device_c64(x), n, batch, 1, n, direction, C64, options={"staged": 1}).cpu().numpy()
+            xin, tol = x.astype(np.complex128), TOL32
+        else:
+            h = inputs.to_half_storage(x)
+            got = half_to_c128(run_fft(to_device_half(h), n, batch, 1, n, direction, C32H, options={"staged": 1}))
+            xin, tol = inputs.from_half_storage(h), TOL16
+        want = oracle.fft_rows(xin[rows], direction)
+        assert max(worst_rel_l2(got[rows], want)) <= tol
+        assert np.isfinite(np.abs(got)).all()
+    assert B.tma_timeouts() == 0
+
+
+def test_staged_rows_default_choice_and_other_sizes():
+    """fp16 storage at n = 16384 takes the staged kernel by default once every multiprocessor
+    has two transforms: same network, so the result equals the plain kernel's bit for bit.
+    Sizes without a staged variant refuse the option and keep working."""
+    import torch
+    from paper_2609_32237_b200 import binding as B
+    n, batch = 16384, 300
+    h = inputs.to_half_storage(inputs.gaussian_complex64((batch, n), 77))
+    a = run_fft(to_device_half(h), n, batch, 1, n, FWD, C32H).cpu().numpy()
+    b = run_fft(to_device_half(h), n, batch, 1, n, FWD, C32H, options={"staged": 0}).cpu().numpy()
+    assert np.array_equal(a.view(np.uint16), b.view(np.uint16))
+    plan = B.fft_plan_create(4096, 8, 1, 4096, FWD, C64)
+    try:
+        with pytest.raises(B.B200FftError) as e:
+            B.fft_plan_set_option(plan, "staged", 1)
+        assert e.value.status == 2
+        x4 = inputs.gaussian_complex64((8, 4096), 5)                 # the plan still works afterwards
+        d = to_device_c64(x4)
+        o = torch.zeros_like(d)
+        B.fft_execute(plan, d.data_ptr(), o.data_ptr(), torch.cuda.current_stream().cuda_stream)
+        torch.cuda.synchronize()
+        assert max(worst_rel_l2(o.cpu().numpy(), oracle.fft_rows(x4.astype(np.complex128), FWD))) <= TOL32
+    finally:
+        B.fft_plan_destroy(plan)
+    assert B.tma_timeouts() == 0
