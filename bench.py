@@ -388,6 +388,26 @@ def run_others(torch, B, args, peak):
         out[name] = s
         torch.cuda.empty_cache()
 
+    # the copy rate of this very device in this very run, beside the stored peak (context only:
+    # the roofline denominators stay the stored measurements)
+    stream = torch.cuda.current_stream()
+    src = torch.empty(1 << 30, dtype=torch.uint8, device="cuda").fill_(1)
+    dst = torch.empty_like(src)
+    per = []
+    for i in range(warmup + steps):
+        flush_l2(torch, scratch)
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        dst.copy_(src)
+        b.record(stream)
+        torch.cuda.synchronize()
+        if i >= warmup:
+            per.append(a.elapsed_time(b))
+    out["device_copy_1gib"] = summarize(per, 2 << 30, peak)
+    out["device_copy_1gib"]["note"] = "device-to-device copy of 1 GiB (1 GiB read + 1 GiB written), same protocol"
+    del src, dst
+    torch.cuda.empty_cache()
+
     fft_case("fft_n4096_b32768_c64_inverse", 4096, 32768, 0, 1, direction=1)
     fft_case("fft_n8192_b16384_c64", 8192, 16384, 0, 2)
     fft_case("fft_n16384_b8192_c64", 16384, 8192, 0, 2)
