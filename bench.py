@@ -381,8 +381,9 @@ def run_others(torch, B, args, peak):
     scratch = torch.empty(512 << 20, dtype=torch.uint8, device="cuda")
     out = {}
 
-    def fft_case(name, n, batch, dtype, seed, layout="rows", direction=-1):
-        _, per, _ = bench_fft(torch, B, n, batch, dtype, seed, steps, warmup, layout, direction, cold_flush=scratch)
+    def fft_case(name, n, batch, dtype, seed, layout="rows", direction=-1, options=None):
+        _, per, _ = bench_fft(torch, B, n, batch, dtype, seed, steps, warmup, layout, direction, cold_flush=scratch,
+                              options=options)
         s = summarize(per, metrics.fft_bytes(n, batch, dtype), peak)
         s["gflops"] = metrics.fft_gflops(n, batch, s["ms_median"] * 1e-3)
         out[name] = s
@@ -416,6 +417,9 @@ def run_others(torch, B, args, peak):
     fft_case("fft_n1024_b256_c64", 1024, 256, 0, 0)
     fft_case("fft_cols_4096x4096_c64", 4096, 4096, 0, 3, layout="cols")
     fft_case("fft_n65536_b2048_c64_four_step", 65536, 2048, 0, 5)
+    fft_case("fft_cols_4096x4096_c64_via_transpose", 4096, 4096, 0, 3, layout="cols", options={"via_transpose": 1})
+    out["fft_cols_4096x4096_c64_via_transpose"]["note"] = ("the paper's four-pass form as a comparison: transpose, row "
+                                                           "transforms, transpose back (three passes; bytes counted once)")
     out["fft_n65536_b2048_c64_four_step"]["note"] = "two passes: algorithmic bytes counted once (16 B/point)"
 
     # 2-D: rows then columns, in place

@@ -116,7 +116,14 @@ int fft_plan_destroy(fft_plan_t plan);
  * 0 forbids it, -1 restores the default (on for fp16 storage with a batch of
  * at least two transforms per multiprocessor); B200FFT_ERR_UNSUPPORTED for
  * other sizes; same results. Every wait on such a copy is bounded:
- * b200fft_tma_timeouts() counts waits that gave up. Unknown keys return
+ * b200fft_tma_timeouts() counts waits that gave up. Key "via_transpose" value
+ * 1 makes a columns plan work the way the paper's four-pass pipeline does
+ * (Section "End to End": a transpose, then the transform along rows) instead
+ * of reading the columns directly: transpose into the workspace, row
+ * transforms in place there, transpose back into `out`; it then needs a
+ * workspace of n*batch elements of the storage type (set_workspace), which
+ * must be neither `in` nor `out`; same results; kept as a measured comparison
+ * with the direct column kernel. Unknown keys return
  * B200FFT_ERR_INVALID_ARG. Must be called before set_workspace. */
 int fft_plan_set_option(fft_plan_t plan, const char *key, int64_t value);
 

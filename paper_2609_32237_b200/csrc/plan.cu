@@ -21,6 +21,9 @@ struct b200fft_plan_s {
     bool four_step;
     int cluster;                 // CTAs per tile requested by the "cluster" option (0 = default)
     int prefetch_ahead;          // "prefetch" option: tiles ahead to prefetch into L2 (-1 = default)
+    bool via_transpose;          // "via_transpose" option (columns): transpose, row transforms, transpose back
+    const KernelEntry* rows_kernel;   // its row variant and table
+    float2* tw_rows;
     int staged;                  // "staged" option: persistent kernel fed by the copy engine (-1 = default)
     const KernelEntry* kernel;   // single-pass variant
     float2* tw;                  // its twiddle rows (device)
@@ -71,6 +74,8 @@ static int build_single_pass(b200fft_plan_s* p) {
 static void release(b200fft_plan_s* p) {
     if (p->tw) cudaFree(p->tw);
     p->tw = nullptr;
+    if (p->tw_rows) cudaFree(p->tw_rows);
+    p->tw_rows = nullptr;
     fourstep_release(&p->fs);
     if (p->pipe_ready) {
         cudaStreamDestroy(p->s_in);
@@ -169,6 +174,27 @@ extern "C" int fft_plan_set_option(fft_plan_t p, const char* key, int64_t value)
         p->prefetch_ahead = (int)value;
         return B200FFT_OK;
     }
+    if (std::strcmp(key, "via_transpose") == 0) {
+        if (p->four_step || p->layout != LAYOUT_COLS) return B200FFT_ERR_UNSUPPORTED;
+        if (!value) {
+            p->via_transpose = false;
+            return B200FFT_OK;
+        }
+        if (!p->rows_kernel) {
+            const KernelEntry* k = find_rows_kernel((int)p->n, p->direction == B200FFT_INVERSE, p->dtype, p->dtype, 0, p->batch);
+            if (!k || k->cl == 1017) k = find_rows_kernel((int)p->n, p->direction == B200FFT_INVERSE, p->dtype, p->dtype, 1, p->batch);
+            if (!k) return B200FFT_ERR_UNSUPPORTED;
+            if (cudaMalloc(&p->tw_rows, sizeof(float2) * (size_t)k->tw_total) != cudaSuccess) {
+                cudaGetLastError();
+                p->tw_rows = nullptr;
+                return B200FFT_ERR_ALLOC;
+            }
+            if (k->build_tw(p->tw_rows, 0) != cudaSuccess || cudaStreamSynchronize(0) != cudaSuccess) return B200FFT_ERR_CUDA;
+            p->rows_kernel = k;
+        }
+        p->via_transpose = true;
+        return B200FFT_OK;
+    }
     if (std::strcmp(key, "staged") == 0) {
         if (p->four_step || p->layout != LAYOUT_ROWS || value < -1 || value > 1) return B200FFT_ERR_UNSUPPORTED;
         const int old = p->staged;
@@ -208,7 +234,7 @@ extern "C" int fft_plan_set_option(fft_plan_t p, const char* key, int64_t value)
 
 extern "C" int fft_plan_workspace_bytes(fft_plan_t p, size_t* bytes) {
     if (!p || !bytes) return B200FFT_ERR_INVALID_ARG;
-    *bytes = p->four_step ? (size_t)p->n * (size_t)p->batch * (size_t)elem_bytes(p->dtype) : 0;
+    *bytes = (p->four_step || p->via_transpose) ? (size_t)p->n * (size_t)p->batch * (size_t)elem_bytes(p->dtype) : 0;
     return B200FFT_OK;
 }
 
@@ -234,6 +260,28 @@ extern "C" int fft_execute(fft_plan_t p, const void* in, void* out, void* stream
         fft_plan_workspace_bytes(p, &need);
         if (!p->workspace || p->workspace_bytes < need) return B200FFT_ERR_WORKSPACE;
         return fourstep_execute(&p->fs, in, out, p->workspace, st);
+    }
+    if (p->via_transpose) {
+        size_t need = 0;
+        fft_plan_workspace_bytes(p, &need);
+        if (!p->workspace || p->workspace_bytes < need) return B200FFT_ERR_WORKSPACE;
+        if (p->workspace == in || p->workspace == out) return B200FFT_ERR_INVALID_ARG;
+        const int eb = elem_bytes(p->dtype);
+        // [n][batch] (row pitch stride) -> [batch][n], transform the rows in place, and back
+        if (transpose_launch(in, p->workspace, (int)p->n, (int)p->batch, p->stride, p->n, eb, st) != cudaSuccess)
+            return B200FFT_ERR_CUDA;
+        FftArgs a;
+        a.in = p->workspace;
+        a.out = p->workspace;
+        a.tw = p->tw_rows;
+        a.prefetch_ahead = 0;
+        a.scale = (p->direction == B200FFT_INVERSE) ? (float)(1.0 / (double)p->n) : 1.0f;
+        a.tiles = p->batch;
+        a.dist = p->n;
+        if (p->rows_kernel->launch(a, st) != cudaSuccess) return B200FFT_ERR_CUDA;
+        if (transpose_launch(p->workspace, out, (int)p->batch, (int)p->n, p->n, p->stride, eb, st) != cudaSuccess)
+            return B200FFT_ERR_CUDA;
+        return B200FFT_OK;
     }
     return launch_single_pass(p, in, out, p->layout == LAYOUT_ROWS ? p->batch : p->batch / p->kernel->w, st);
 }

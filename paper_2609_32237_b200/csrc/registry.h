@@ -87,6 +87,9 @@ constexpr KernelEntry make_entry() {
 const KernelEntry* find_rows_kernel(int n, bool inverse, int in_dtype, int out_dtype, int cl = 0,
                                     int64_t batch = (int64_t)1 << 40);
 const KernelEntry* find_cols_kernel(int n, bool inverse, int in_dtype, int out_dtype, int cl = 0);
+// out[c * ld_out + r] = in[r * ld_in + c]; elem_bytes 8 (complex64) or 4 (complex half)
+cudaError_t transpose_launch(const void* in, void* out, int rows, int cols, int64_t ld_in, int64_t ld_out, int elem_bytes,
+                             cudaStream_t st);
 int tma_timeouts();   // mbarrier waits of the TMA column variant that ran out of polls since load
 int rows_stage_timeouts();   // the same for the staged persistent row kernels
 

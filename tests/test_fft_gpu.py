@@ -427,3 +427,42 @@ def test_staged_rows_default_choice_and_other_sizes():
     finally:
         B.fft_plan_destroy(plan)
     assert B.tma_timeouts() == 0
+
+
+@pytest.mark.parametrize("n,cols,ld", [(1024, 24, 24), (4096, 68, 72), (256, 36, 40)])
+def test_columns_via_transpose(n, cols, ld):
+    """A columns plan run as transpose + row transforms + transpose back (the paper's four-pass
+    form): same results as the oracle and as the direct column kernel, padding untouched,
+    both storage types and directions; the workspace is required."""
+    import torch
+    from paper_2609_32237_b200 import binding as B
+    m = inputs.uniform_complex64((n, ld), 61)
+    for direction in (FWD, INV):
+        want = oracle.fft_cols(m[:, :cols].astype(np.complex128), direction)
+        got = run_fft(to_device_c64(m), n, cols, ld, 1, direction, C64, options={"via_transpose": 1}).cpu().numpy()
+        direct = run_fft(to_device_c64(m), n, cols, ld, 1, direction, C64).cpu().numpy()
+        per_col = np.linalg.norm(got[:, :cols] - want, axis=0) / np.linalg.norm(want, axis=0)
+        assert per_col.max() <= TOL32
+        assert rel_l2(got[:, :cols], direct[:, :cols]) <= 1e-6
+        assert np.all(got[:, cols:] == 0)
+    h = inputs.to_half_storage(m)
+    want = oracle.fft_cols(inputs.from_half_storage(h)[:, :cols], FWD)
+    got = half_to_c128(run_fft(to_device_half(h), n, cols, ld, 1, FWD, C32H, options={"via_transpose": 1}))
+    assert rel_l2(got[:, :cols], want) <= TOL16
+    plan = B.fft_plan_create(n, cols, ld, 1, FWD, C64)
+    try:
+        B.fft_plan_set_option(plan, "via_transpose", 1)
+        assert B.fft_plan_workspace_bytes(plan) == n * cols * 8
+        d = to_device_c64(m)
+        with pytest.raises(B.B200FftError) as e:
+            B.fft_execute(plan, d.data_ptr(), d.data_ptr(), torch.cuda.current_stream().cuda_stream)
+        assert e.value.status == 6
+    finally:
+        B.fft_plan_destroy(plan)
+    rows_plan = B.fft_plan_create(n, 4, 1, n, FWD, C64)
+    try:
+        with pytest.raises(B.B200FftError) as e:
+            B.fft_plan_set_option(rows_plan, "via_transpose", 1)
+        assert e.value.status == 2
+    finally:
+        B.fft_plan_destroy(rows_plan)
