@@ -55,10 +55,16 @@ static int build_single_pass(b200fft_plan_s* p) {
         const bool by_default = p->n == 16384 && p->dtype == B200FFT_C32H && p->batch >= 2 * (int64_t)p->sms;
         if (p->staged == 1 || (p->staged == -1 && by_default)) cl = 1017;
     }
-    const KernelEntry* k = (p->layout == LAYOUT_ROWS)
-                               ? find_rows_kernel((int)p->n, inv, p->dtype, p->dtype, cl, p->batch)
-                               : find_cols_kernel((int)p->n, inv, p->dtype, p->dtype, cl);
+    const KernelEntry* k = nullptr;
+    if (p->layout == LAYOUT_COLS && cl == 0) {          // wide tiles where they exist and divide the batch
+        k = find_cols_kernel((int)p->n, inv, p->dtype, p->dtype, 1019);
+        if (k && p->batch % k->w) k = nullptr;
+    }
+    if (!k)
+        k = (p->layout == LAYOUT_ROWS) ? find_rows_kernel((int)p->n, inv, p->dtype, p->dtype, cl, p->batch)
+                                       : find_cols_kernel((int)p->n, inv, p->dtype, p->dtype, cl);
     if (!k) return B200FFT_ERR_UNSUPPORTED;
+    if (p->layout == LAYOUT_COLS && p->batch % k->w) return B200FFT_ERR_UNSUPPORTED;
     p->kernel = k;                  // the table depends on the factorisation: always rebuilt
     if (p->tw) cudaFree(p->tw);
     p->tw = nullptr;

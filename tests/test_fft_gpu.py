@@ -466,3 +466,23 @@ def test_columns_via_transpose(n, cols, ld):
         assert e.value.status == 2
     finally:
         B.fft_plan_destroy(rows_plan)
+
+
+@pytest.mark.parametrize("n,cols,ld", [(256, 32, 40), (512, 16, 16), (1024, 24, 24), (1024, 40, 48)])
+def test_columns_wide_tiles_by_default(n, cols, ld):
+    """Short column transforms whose batch is a multiple of the wide tile (16 columns, 8 at
+    n = 1024) take it by default: checked against the oracle and the narrow-tile kernel
+    (option cluster = 1), both directions and storage types, padding untouched."""
+    m = inputs.uniform_complex64((n, ld), 62)
+    for direction in (FWD, INV):
+        want = oracle.fft_cols(m[:, :cols].astype(np.complex128), direction)
+        got = run_fft(to_device_c64(m), n, cols, ld, 1, direction, C64).cpu().numpy()
+        narrow = run_fft(to_device_c64(m), n, cols, ld, 1, direction, C64, options={"cluster": 1}).cpu().numpy()
+        per_col = np.linalg.norm(got[:, :cols] - want, axis=0) / np.linalg.norm(want, axis=0)
+        assert per_col.max() <= TOL32
+        assert rel_l2(got[:, :cols], narrow[:, :cols]) <= 1e-6
+        assert np.all(got[:, cols:] == 0)
+    h = inputs.to_half_storage(m)
+    want = oracle.fft_cols(inputs.from_half_storage(h)[:, :cols], FWD)
+    got = half_to_c128(run_fft(to_device_half(h), n, cols, ld, 1, FWD, C32H))
+    assert rel_l2(got[:, :cols], want) <= TOL16
