@@ -60,7 +60,8 @@ class ClockSampler:
         self.index = index
         self.proc = None
         self.lines = []
-        self.samples = []          # (sm_mhz, reasons bitmask)
+        self.samples = []          # (time, sm_mhz, reasons bitmask)
+        self.window = [None, None]  # timed region, time.monotonic()
         self.max_mhz = None
         self.nvml = None
         self.stop_flag = False
@@ -103,14 +104,20 @@ class ClockSampler:
                     rs = int(n.nvmlDeviceGetCurrentClocksEventReasons(self.handle))
                 except Exception:
                     rs = int(n.nvmlDeviceGetCurrentClocksThrottleReasons(self.handle))
-                self.samples.append((mhz, rs))
+                self.samples.append((time.monotonic(), mhz, rs))
             except Exception:
                 pass
             time.sleep(0.002)
 
+    def mark_begin(self):
+        self.window[0] = time.monotonic()
+
+    def mark_end(self):
+        self.window[1] = time.monotonic()
+
     def _read(self):
         for line in self.proc.stdout:
-            self.lines.append(line.strip())
+            self.lines.append((time.monotonic(), line.strip()))
 
     def stop(self):
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
@@ -119,8 +126,14 @@ class ClockSampler:
             self.thread.join(timeout=1)
             n = self.nvml
             bits = {"hw_slowdown": 0x8, "hw_thermal_slowdown": 0x40, "sw_thermal_slowdown": 0x20, "sw_power_cap": 0x4}
-            reasons = sorted(k for k, b in bits.items() if any(rs & b for _, rs in self.samples))
-            sm = [m for m, _ in self.samples]
+            t0, t1 = self.window
+            inside = [(m, rs) for t, m, rs in self.samples if (t0 is None or t >= t0) and (t1 is None or t <= t1)]
+            if not inside and self.samples:      # a region shorter than one poll: the nearest sample
+                mid = 0.5 * ((t0 or 0.0) + (t1 or 0.0))
+                t, m, rs = min(self.samples, key=lambda x: abs(x[0] - mid))
+                inside = [(m, rs)]
+            reasons = sorted(k for k, b in bits.items() if any(rs & b for _, rs in inside))
+            sm = [m for m, _ in inside]
             return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": self.max_mhz,
                     "sm_min_mhz": float(min(sm)) if sm else None, "reasons": reasons, "samples": len(sm),
                     "source": "nvml, 2 ms polling during the timed region"}
@@ -133,7 +146,11 @@ class ClockSampler:
         except Exception:
             self.proc.kill()
         sm, mx, reasons = [], None, set()
-        for ln in self.lines:
+        t0, t1 = self.window
+        lines = [ln for t, ln in self.lines if (t0 is None or t >= t0 - 0.1) and (t1 is None or t <= t1 + 0.1)]
+        if not lines:
+            lines = [ln for _, ln in self.lines]
+        for ln in lines:
             parts = [p.strip() for p in ln.split(",")]
             if len(parts) < 6:
                 continue
@@ -298,22 +315,24 @@ def run_gpu(args):
     def step():
         B.fft_execute(plan, d_in.data_ptr(), d_out.data_ptr(), stream.cuda_stream)
 
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()                  # polls from before the warm-up; only samples inside the timed window count
     for _ in range(max(args.warmup, 3)):
         step()
     torch.cuda.synchronize()
     if world > 1:
         dist.barrier()
-    sampler = ClockSampler(local)
-    if rank == 0:
-        sampler.start()
     launches0 = B.launch_count()
     torch.cuda.synchronize()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler.mark_begin()
     e0.record(stream)
     for _ in range(args.steps):
         step()
     e1.record(stream)
     torch.cuda.synchronize()
+    sampler.mark_end()
     total_ms = e0.elapsed_time(e1)
     launches = B.launch_count() - launches0
     if world > 1:
