@@ -50,8 +50,8 @@ static int build_single_pass(b200fft_plan_s* p) {
     int cl = p->cluster;
     if (p->layout == LAYOUT_ROWS && cl == 0) {
         // Persistent staged kernel: measured on B200 at n = 16384 with fp16 storage, 379 -> 342 us for
-        // 8192 transforms; with fp32 storage it is slower than the plain kernel (478 against 447 us:
-        // the staged tile leaves the L1 cache 30 KiB), so there it is only taken on request.
+        // 8192 transforms; with fp32 storage it is slower than the plain kernel (455 against 447 us:
+        // only half of the tile can wait beside the exchange buffer), so there it is only taken on request.
         const bool by_default = p->n == 16384 && p->dtype == B200FFT_C32H && p->batch >= 2 * (int64_t)p->sms;
         if (p->staged == 1 || (p->staged == -1 && by_default)) cl = 1017;
     }
