@@ -434,6 +434,26 @@ def run_others(torch, B, args, peak):
     fft_case("fft_n8192_b16384_c32h", 8192, 16384, 1, 2)
     fft_case("fft_n16384_b8192_c32h", 16384, 8192, 1, 2)
     fft_case("fft_n1024_b256_c64", 1024, 256, 0, 0)
+
+    # block floating point on fp16 storage (one exponent per transform): the cost of the maximum search
+    h = torch.from_numpy(inputs.to_half_storage(inputs.gaussian_complex64((16384, 8192), 2))).cuda()
+    ho = torch.empty_like(h)
+    ex = torch.zeros(16384, dtype=torch.int32, device="cuda")
+    pb = B.fft_plan_create(8192, 16384, 1, 8192, -1, 1)
+    per = []
+    for i in range(warmup + steps):
+        flush_l2(torch, scratch)
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        B.fft_execute_bfp(pb, h.data_ptr(), 0, ho.data_ptr(), ex.data_ptr(), stream.cuda_stream)
+        b.record(stream)
+        torch.cuda.synchronize()
+        if i >= warmup:
+            per.append(a.elapsed_time(b))
+    B.fft_plan_destroy(pb)
+    out["fft_n8192_b16384_c32h_block_floating_point"] = summarize(per, metrics.fft_bytes(8192, 16384, 1), peak)
+    del h, ho, ex
+    torch.cuda.empty_cache()
     fft_case("fft_cols_4096x4096_c64", 4096, 4096, 0, 3, layout="cols")
     fft_case("fft_n65536_b2048_c64_four_step", 65536, 2048, 0, 5)
     fft_case("fft_cols_4096x4096_c64_via_transpose", 4096, 4096, 0, 3, layout="cols", options={"via_transpose": 1})

@@ -150,6 +150,24 @@ int fft_plan_set_option(fft_plan_t plan, const char *key, int64_t value);
 #define B200FFT_NOALLOC_MAX_ELEMS 262144
 int fft_execute_noalloc(int64_t n, int64_t batch, int direction, const void *in, void *out, void *stream);
 
+/* Block-floating-point form of fft_execute for rows plans with fp16 storage and
+ * 1024 <= n <= 16384 (paper, Section "FP16 Storage": FFT outputs grow up to N
+ * times for coherent data, so real radar data in fp16 needs block floating
+ * point; the paper's own chain uses fixed shifts, see sar_rda_*). Every
+ * transform b carries one power-of-two exponent:
+ *   true input  x_b[n] = in_b[n]  * 2^in_exp[b]   (in_exp == NULL: all zero)
+ *   true output X_b[k] = out_b[k] * 2^out_exp[b]
+ * The transform is computed in fp32 from the stored fp16 values; the stored
+ * output is scaled by the power of two that puts its largest real or imaginary
+ * component in [2^14, 2^15) (all-zero output: unscaled), and out_exp[b] =
+ * in_exp[b] + that shift (the inverse's 1/n goes into the exponent too).
+ * in_exp, out_exp: device arrays of `batch` int32; in/out as for fft_execute
+ * (in place allowed; in_exp may equal out_exp). No workspace. Errors:
+ * B200FFT_ERR_UNSUPPORTED for other plans, B200FFT_ERR_ALIGNMENT,
+ * B200FFT_ERR_INVALID_ARG for null pointers. */
+int fft_execute_bfp(fft_plan_t plan, const void *in, const int32_t *in_exp, void *out, int32_t *out_exp,
+                    void *stream);
+
 /* Static description of a status code. */
 const char *fft_status_string(int status);
 

@@ -25,6 +25,7 @@ EXPORTS = [
     "b200fft_launch_count", "sar_rda_params_create", "sar_rda_workspace_bytes",
     "sar_rda_set_workspace", "sar_rda_form_image", "sar_rda_form_image_host", "sar_rda_run_step",
     "sar_rda_params_destroy", "fft_execute_noalloc", "sar_rda_set_option", "b200fft_tma_timeouts",
+    "fft_execute_bfp",
 ]
 
 
@@ -69,6 +70,7 @@ def _load():
     L.sar_rda_run_step.argtypes = [vp, vp, vp, ci, vp]
     L.sar_rda_params_destroy.argtypes = [vp]
     L.fft_execute_noalloc.argtypes = [i64, i64, ci, vp, vp, vp]
+    L.fft_execute_bfp.argtypes = [vp, vp, vp, vp, vp, vp]
     L.sar_rda_set_option.argtypes = [vp, ctypes.c_char_p, i64]
     return L
 
@@ -134,6 +136,12 @@ def fft_execute_noalloc(n, batch, direction, in_ptr, out_ptr, stream=0):
 
 
 NOALLOC_MAX_ELEMS = 262144
+
+
+def fft_execute_bfp(plan, in_ptr, in_exp_ptr, out_ptr, out_exp_ptr, stream=0):
+    """Block-floating-point transform of fp16-stored rows: one int32 power-of-two exponent per
+    transform on the way in (0 / None: all zero) and on the way out."""
+    _check(_lib.fft_execute_bfp(plan, in_ptr, in_exp_ptr or None, out_ptr, out_exp_ptr, stream), "fft_execute_bfp")
 
 
 def fft_plan_destroy(plan):

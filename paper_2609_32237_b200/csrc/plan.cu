@@ -24,6 +24,8 @@ struct b200fft_plan_s {
     bool via_transpose;          // "via_transpose" option (columns): transpose, row transforms, transpose back
     const KernelEntry* rows_kernel;   // its row variant and table
     float2* tw_rows;
+    const BfpEntry* bfp;         // block-floating-point variant and its table, built on first use
+    float2* tw_bfp;
     int staged;                  // "staged" option: persistent kernel fed by the copy engine (-1 = default)
     const KernelEntry* kernel;   // single-pass variant
     float2* tw;                  // its twiddle rows (device)
@@ -82,6 +84,8 @@ static void release(b200fft_plan_s* p) {
     p->tw = nullptr;
     if (p->tw_rows) cudaFree(p->tw_rows);
     p->tw_rows = nullptr;
+    if (p->tw_bfp) cudaFree(p->tw_bfp);
+    p->tw_bfp = nullptr;
     fourstep_release(&p->fs);
     if (p->pipe_ready) {
         cudaStreamDestroy(p->s_in);
@@ -290,6 +294,34 @@ extern "C" int fft_execute(fft_plan_t p, const void* in, void* out, void* stream
         return B200FFT_OK;
     }
     return launch_single_pass(p, in, out, p->layout == LAYOUT_ROWS ? p->batch : p->batch / p->kernel->w, st);
+}
+
+extern "C" int fft_execute_bfp(fft_plan_t p, const void* in, const int32_t* in_exp, void* out, int32_t* out_exp,
+                               void* stream) {
+    if (!p || !in || !out || !out_exp) return B200FFT_ERR_INVALID_ARG;
+    if (p->layout != LAYOUT_ROWS || p->dtype != B200FFT_C32H || p->four_step) return B200FFT_ERR_UNSUPPORTED;
+    if (reinterpret_cast<uintptr_t>(in) % 16 || reinterpret_cast<uintptr_t>(out) % 16) return B200FFT_ERR_ALIGNMENT;
+    if (!p->bfp) {
+        const BfpEntry* k = find_bfp_kernel((int)p->n, p->direction == B200FFT_INVERSE);
+        if (!k) return B200FFT_ERR_UNSUPPORTED;
+        if (cudaMalloc(&p->tw_bfp, sizeof(float2) * (size_t)k->tw_total) != cudaSuccess) {
+            cudaGetLastError();
+            p->tw_bfp = nullptr;
+            return B200FFT_ERR_ALLOC;
+        }
+        if (k->build_tw(p->tw_bfp, 0) != cudaSuccess || cudaStreamSynchronize(0) != cudaSuccess) return B200FFT_ERR_CUDA;
+        p->bfp = k;
+    }
+    FftArgs a;
+    a.in = in;
+    a.out = out;
+    a.tw = p->tw_bfp;
+    a.prefetch_ahead = 0;
+    a.scale = 1.0f;
+    a.tiles = p->batch;
+    a.dist = p->dist;
+    return p->bfp->launch(a, in_exp, out_exp, reinterpret_cast<cudaStream_t>(stream)) == cudaSuccess ? B200FFT_OK
+                                                                                                      : B200FFT_ERR_CUDA;
 }
 
 // one launch of the plan's single-pass kernel over `tiles` tiles starting at in/out

@@ -83,6 +83,16 @@ constexpr KernelEntry make_entry() {
     make_entry<C, false, StoreC32H, StoreC32H>(),           \
     make_entry<C, true, StoreC32H, StoreC32H>()
 
+// block-floating-point row transforms (fp16 storage, one exponent per transform)
+struct BfpEntry {
+    int n;
+    bool inverse;
+    int tw_total;
+    cudaError_t (*launch)(const FftArgs&, const int* in_exp, int* out_exp, cudaStream_t);
+    cudaError_t (*build_tw)(float2*, cudaStream_t);
+};
+const BfpEntry* find_bfp_kernel(int n, bool inverse);
+
 // cl: CTAs per tile (cluster size); 0 picks the default variant for that size
 const KernelEntry* find_rows_kernel(int n, bool inverse, int in_dtype, int out_dtype, int cl = 0,
                                     int64_t batch = (int64_t)1 << 40);
