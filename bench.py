@@ -166,6 +166,64 @@ class ClockSampler:
                 "reasons": sorted(reasons), "samples": len(sm), "source": "nvidia-smi -lms 100"}
 
 
+def run_landscape(args):
+    """Throughput against transform size, N = 32 ... 2^20 (the paper's Figure "landscape", our
+    kernels only): cold on a 1 GiB footprint (512 MiB in + 512 MiB out, a 512 MiB scratch write
+    before every sample) and hot on a 32 MiB footprint that stays in the 126 MB L2."""
+    import torch
+    torch.cuda.set_device(0)
+    from paper_2609_32237_b200 import binding as B
+    peak, _ = measured_peak_gbs()
+    stream = torch.cuda.current_stream()
+    scratch = torch.empty(512 << 20, dtype=torch.uint8, device="cuda")
+    big = torch.randn(1 << 26, 2, device="cuda")
+    big_out = torch.empty_like(big)
+    rows = []
+    for lg in range(5, 21):
+        n = 1 << lg
+        row = {"n": n}
+        for label, points, cold in (("cold_1gib", 1 << 26, True), ("hot_32mib", 1 << 21, False)):
+            batch = points // n
+            plan = B.fft_plan_create(n, batch, 1, n, -1, 0)
+            need = B.fft_plan_workspace_bytes(plan)
+            ws = None
+            if need:
+                ws = torch.empty(need, dtype=torch.uint8, device="cuda")
+                B.fft_plan_set_workspace(plan, ws.data_ptr(), need)
+            call = lambda: B.fft_execute(plan, big.data_ptr(), big_out.data_ptr(), stream.cuda_stream)
+            for _ in range(3):
+                call()
+            torch.cuda.synchronize()
+            nb = metrics.fft_bytes(n, batch, 0)
+            if cold:
+                per = []
+                for _ in range(9):
+                    flush_l2(torch, scratch)
+                    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    a.record(stream)
+                    call()
+                    b.record(stream)
+                    torch.cuda.synchronize()
+                    per.append(a.elapsed_time(b))
+                ms = float(np.median(per))
+            else:
+                reps = 200
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(stream)
+                for _ in range(reps):
+                    call()
+                b.record(stream)
+                torch.cuda.synchronize()
+                ms = a.elapsed_time(b) / reps
+            B.fft_plan_destroy(plan)
+            del ws
+            row[label] = {"batch": batch, "us": ms * 1e3, "gbs": nb / ms / 1e6,
+                          "gflops": metrics.fft_gflops(n, batch, ms * 1e-3)}
+        rows.append(row)
+    print(json.dumps({"landscape": "complex64 forward rows, N = 32 ... 2^20", "hbm_peak_gbs": peak, "rows": rows}))
+    return 0
+
+
 def dist_env():
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -630,10 +688,13 @@ def main():
                     help="run one workload only, e.g. rows:16384:8192:c64, cols:4096:4096:c64, sar:c64")
     ap.add_argument("--option", action="append", default=[],
                     help="with --case rows/cols: plan option KEY=VALUE (repeatable), e.g. cluster=4")
+    ap.add_argument("--landscape", action="store_true", help="throughput against N = 32 ... 2^20, cold 1 GiB and hot 32 MiB")
     ap.add_argument("--sweep", action="store_true", help="hot vs cold throughput against the batch footprint")
     args = ap.parse_args()
     if args.sweep:
         return run_sweep(args)
+    if args.landscape:
+        return run_landscape(args)
     if args.case:
         return run_case(args)
     if args.impl == "reference":
