@@ -56,9 +56,11 @@ typedef struct b200fft_sar_s *sar_rda_params_t;
  *   columns  dist == 1, stride >= batch, stride and batch even: the columns of
  *            a row-major matrix (paper, Section "End to End": the FFT that
  *            reads the columns directly)
- * Supported sizes: n a power of two, 32 <= n <= 16384 in a single pass over
- * memory (columns: 256 <= n <= 8192); 2^15 <= n <= 2^20 (rows only) by a two-pass four-step split (the
- * paper's "usual remedy when a transform does not fit on chip"), which needs a
+ * Supported sizes: n a power of two, 32 <= n <= 32768 in a single pass over
+ * memory (columns: 256 <= n <= 8192; rows of n = 32768 on a cluster of two
+ * thread blocks that share the transform through distributed shared memory);
+ * 2^16 <= n <= 2^20 (rows only) by a two-pass four-step split (the paper's
+ * "usual remedy when a transform does not fit on chip"), which needs a
  * workspace of n*batch elements of the storage type.
  *
  * fft_plan_create allocates the plan's twiddle tables on the current device
@@ -100,7 +102,8 @@ int fft_plan_destroy(fft_plan_t plan);
 
 /* Test knob: force a kernel variant (paper, Section "One Pass": "a regression
  * test forces N=8192 through this path"). key "four_step" value 1 routes a
- * rows plan of any supported n >= 4096 through the two-pass split. Key
+ * rows plan of any supported n >= 4096 through the two-pass split (value 0
+ * brings a plan of n <= 32768 back to its single pass). Key
  * "cluster" value c (1, 2 or 4; 0 = the default for that size) picks the
  * variant of a single-pass plan in which c CTAs of one thread-block cluster
  * share a tile through distributed shared memory; B200FFT_ERR_UNSUPPORTED if

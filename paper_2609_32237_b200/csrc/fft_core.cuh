@@ -213,7 +213,7 @@ struct Cfg {
     // registers per thread are capped at 128 so that at least 65536 / (128 * THREADS) CTAs fit an SM
     static constexpr int MINB = (65536 / (128 * THREADS)) > 0 ? (65536 / (128 * THREADS)) : 1;
     static_assert(P_ % R1_ == 0 && P_ % R2_ == 0 && P_ % R3_ == 0 && P_ % R4_ == 0, "P must be a multiple of every radix");
-    static_assert(P_ / radix(S) >= 2, "the last stage needs two butterflies per thread (128-bit stores)");
+    static_assert(P_ / radix(S) >= 2 || W_ == 1, "column tiles need two butterflies per thread in the last stage");
     static_assert((N_ * W_) % (P_ * CL_) == 0, "tile must divide among threads");
 };
 
@@ -599,6 +599,17 @@ struct Engine {
         using G = Geo<C, S>;
         constexpr int V = G::V, r = G::r;
         constexpr int KS = C::N / r;
+        if constexpr (V == 1) {     // one butterfly per thread: 64-bit stores, one contiguous run per warp
+            int b0, q;
+            last_index(0, b0, q);
+            static_for<0, r>([&](auto j_) {
+                constexpr int j = decltype(j_)::value;
+                float2 a = x[j];
+                if constexpr (CONJ) a.y = -a.y;
+                if constexpr (SCALE) a = make_float2(a.x * scale, a.y * scale);
+                ST::store1(out, base + j * KS + b0, a);
+            });
+        }
         static_for<0, V / 2>([&](auto h_) {
             constexpr int v = 2 * decltype(h_)::value;
             int b0, q;

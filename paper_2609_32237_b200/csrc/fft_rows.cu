@@ -179,6 +179,7 @@ static const KernelEntry k_rows[] = {
     B200FFT_ENTRIES_STD(R8192), B200FFT_ENTRIES_STD(R16384),
     B200FFT_ENTRIES_STD(R8192x2), B200FFT_ENTRIES_STD(R8192x4),
     B200FFT_ENTRIES_STD(R16384x2), B200FFT_ENTRIES_STD(R16384x4),
+    B200FFT_ENTRIES_STD(R32768x2),
 };
 
 static const KernelEntry k_rows_alt[] = {B200FFT_ENTRIES_STD(R4096t15), B200FFT_ENTRIES_STD(R16384s4)};
@@ -188,6 +189,7 @@ static const KernelEntry k_rows_alt[] = {B200FFT_ENTRIES_STD(R4096t15), B200FFT_
 // memory. Measured on B200: n = 16384, batch <= 32: 14.3 -> 10.2 us with 4 CTAs per transform;
 // n = 8192, batch <= 16: 12.3 -> 10.2 us with 2. Large batches are faster with one CTA.
 static int default_cluster(int n, int64_t batch) {
+    if (n == 32768) return 2;
     if (n == 16384 && batch <= 32) return 4;
     if (n == 8192 && batch <= 16) return 2;
     return 1;

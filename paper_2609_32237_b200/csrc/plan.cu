@@ -143,7 +143,9 @@ extern "C" int fft_plan_create(fft_plan_t* plan, int64_t n, int64_t batch, int64
     cudaDeviceGetAttribute(&p->sms, cudaDevAttrMultiProcessorCount, p->device);
 
     int rc;
-    if (n > 16384) {
+    if (n == 32768 && layout == LAYOUT_ROWS) {
+        rc = build_single_pass(p);              // one pass on a cluster of two CTAs; "four_step" = 1 for the split
+    } else if (n > 16384) {
         if (layout != LAYOUT_ROWS) { delete p; return B200FFT_ERR_UNSUPPORTED; }
         p->four_step = true;
         rc = fourstep_build(&p->fs, n, batch, dist, direction, storage_dtype);
@@ -170,7 +172,7 @@ extern "C" int fft_plan_set_option(fft_plan_t p, const char* key, int64_t value)
             p->four_step = true;
             p->workspace = nullptr;
             p->workspace_bytes = 0;
-        } else if (!value && p->four_step && p->n <= 16384) {
+        } else if (!value && p->four_step && p->n <= 32768) {
             if (!p->kernel) {
                 int rc = build_single_pass(p);
                 if (rc != B200FFT_OK) return rc;

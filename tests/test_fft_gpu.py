@@ -166,7 +166,7 @@ def test_config3_columns_and_2d_full():
     assert rel_l2(d.cpu().numpy(), want2d) <= TOL32
 
 
-@pytest.mark.parametrize("n", [4096, 8192, 16384])
+@pytest.mark.parametrize("n", [4096, 8192, 16384, 32768])
 @pytest.mark.parametrize("direction", [FWD, INV])
 def test_four_step_forced_at_single_pass_sizes(n, direction):
     """The two-pass split forced at sizes the single-pass kernels also cover
@@ -486,3 +486,32 @@ def test_columns_wide_tiles_by_default(n, cols, ld):
     want = oracle.fft_cols(inputs.from_half_storage(h)[:, :cols], FWD)
     got = half_to_c128(run_fft(to_device_half(h), n, cols, ld, 1, FWD, C32H))
     assert rel_l2(got[:, :cols], want) <= TOL16
+
+
+def test_n32768_runs_in_one_pass_on_a_cluster_of_two():
+    """n = 32768 does not fit one CTA; by default two CTAs of a cluster share the transform
+    through distributed shared memory, in one pass and without a workspace. Checked against
+    the oracle and the two-pass split, ragged batch, both directions and storage types."""
+    from paper_2609_32237_b200 import binding as B
+    n, batch = 32768, 7
+    plan = B.fft_plan_create(n, batch, 1, n, FWD, C64)
+    try:
+        assert B.fft_plan_workspace_bytes(plan) == 0
+        B.fft_plan_set_option(plan, "four_step", 1)
+        assert B.fft_plan_workspace_bytes(plan) == n * batch * 8
+        B.fft_plan_set_option(plan, "four_step", 0)
+        assert B.fft_plan_workspace_bytes(plan) == 0
+    finally:
+        B.fft_plan_destroy(plan)
+    x = inputs.gaussian_complex64((batch, n + 6), 321)[:, :]
+    for direction in (FWD, INV):
+        want = oracle.fft_rows(x[:, :n].astype(np.complex128), direction)
+        got = run_fft(to_device_c64(x), n, batch, 1, n + 6, direction, C64).cpu().numpy()       # padded rows
+        two = run_fft(to_device_c64(x), n, batch, 1, n + 6, direction, C64, options={"four_step": 1}).cpu().numpy()
+        assert max(worst_rel_l2(got[:, :n], want)) <= TOL32
+        assert rel_l2(got[:, :n], two[:, :n]) <= 1e-6
+        assert np.all(got[:, n:] == 0)
+    h = inputs.to_half_storage(np.ascontiguousarray(x[:, :n]))
+    want = oracle.fft_rows(inputs.from_half_storage(h), FWD)
+    got = half_to_c128(run_fft(to_device_half(h), n, batch, 1, n, FWD, C32H))
+    assert max(worst_rel_l2(got, want)) <= TOL16
