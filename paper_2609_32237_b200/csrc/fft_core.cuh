@@ -206,6 +206,9 @@ struct Cfg {
     static_assert(R1_ * R2_ * R3_ * R4_ == N_, "radices must multiply to N");
     // bits of the element index the swizzle may flip: bits 1..3, but only below the top digit
     static constexpr int SWZ = 14 & (L(1) * W_ - 1);
+    // with one butterfly per thread in the last stage neighbouring lanes hold neighbouring butterflies (not
+    // every other one), so the index is doubled before it is folded into bits 1..3
+    static constexpr int SWM = (P_ / radix(S) == 1) ? 2 : 1;
     static_assert(L(1) * W_ >= 2, "at least two elements below the top digit");
     static_assert(CL_ == 1 || G_ == 1, "a cluster works on one tile");
     static_assert(CL_ >= 1 && R1_ % CL_ == 0 && RC >= 2, "the cluster splits the top digit");
@@ -276,12 +279,12 @@ struct Geo {
     __device__ __forceinline__ int elem() const {
         if constexpr (s == 1) {
             constexpr int jl = j % RC;                // top digit relative to the owner
-            return (e0 + jl * estep) ^ (((bl0 + jl) * W) & C::SWZ);
+            return (e0 + jl * estep) ^ (((bl0 + jl) * W * C::SWM) & C::SWZ);
         } else if constexpr (!last) {
-            if constexpr (C::blw(s) < 16) return (e0 + j * estep) ^ (((bl0 + j * C::blw(s)) * W) & C::SWZ);
-            else return (e0 + j * estep) ^ ((bl0 * W) & C::SWZ);
+            if constexpr (C::blw(s) < 16) return (e0 + j * estep) ^ (((bl0 + j * C::blw(s)) * W * C::SWM) & C::SWZ);
+            else return (e0 + j * estep) ^ ((bl0 * W * C::SWM) & C::SWZ);
         } else {
-            return (e0 + j * estep) ^ ((bl0 * W) & C::SWZ);
+            return (e0 + j * estep) ^ ((bl0 * W * C::SWM) & C::SWZ);
         }
     }
 };
@@ -693,13 +696,16 @@ __global__ void __launch_bounds__(C::THREADS, C::MINB) fft_kernel(const FftArgs 
     const int64_t base = (C::W == 1) ? tile * a.dist : tile * C::W;
     Engine<C> e;
     e.setup(t);
-    if constexpr (C::W == 1 && C::CL == 1 && C::G == 1) {
+    if constexpr (C::W == 1 && C::G == 1) {
         // A large tile leaves room for one or two CTAs per SM, so nothing overlaps this CTA's
         // load phase. One thread asks L2 for the input of the tile that will run where this
-        // one runs now, some CTAs later; that tile's loads then hit L2.
+        // one runs now, some CTAs later; that tile's loads then hit L2. (Each CTA of a cluster
+        // asks for its share of the transform.)
+        constexpr unsigned SHARE = (unsigned)(C::N / C::CL * TIn::ELEM_BYTES);
         if (a.prefetch_ahead > 0 && threadIdx.x == 0 && tile + a.prefetch_ahead < a.tiles)
-            prefetch_l2_bulk(reinterpret_cast<const char*>(a.in) + (tile + a.prefetch_ahead) * a.dist * TIn::ELEM_BYTES,
-                             (unsigned)(C::N * TIn::ELEM_BYTES));
+            prefetch_l2_bulk(reinterpret_cast<const char*>(a.in) + (tile + a.prefetch_ahead) * a.dist * TIn::ELEM_BYTES +
+                                 (size_t)e.rank * SHARE,
+                             SHARE);
     }
     e.template load_first<TIn, INV>(a.in, base, a.dist);
     e.dif(sm, a.tw);

@@ -333,12 +333,12 @@ static int launch_single_pass(b200fft_plan_s* p, const void* in, void* out, int6
     a.out = out;
     a.tw = p->tw;
     a.prefetch_ahead = 0;
-    if (p->layout == LAYOUT_ROWS && p->kernel->cl == 1 && p->kernel->g == 1) {
+    if (p->layout == LAYOUT_ROWS && p->kernel->cl >= 1 && p->kernel->cl <= 8 && p->kernel->g == 1) {
         // default: for tiles that fill an SM (one CTA resident), the tile one full wave ahead;
         // measured on B200: +13 % at n = 16384 rows, nothing to gain at n = 8192 and below,
         // and a loss for column tiles (their time goes to the lock-step compute, not the load)
         const bool fills_sm = p->kernel->smem_bytes > 100 * 1024;
-        a.prefetch_ahead = (p->prefetch_ahead >= 0) ? p->prefetch_ahead : (fills_sm ? p->sms : 0);
+        a.prefetch_ahead = (p->prefetch_ahead >= 0) ? p->prefetch_ahead : (fills_sm ? p->sms / p->kernel->cl : 0);
     }
     a.scale = (p->direction == B200FFT_INVERSE) ? (float)(1.0 / (double)p->n) : 1.0f;
     a.tiles = tiles;
