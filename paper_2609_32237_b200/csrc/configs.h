@@ -25,8 +25,8 @@ using R16384s4 = Cfg<16384, 1, 32, 1, 1, 16, 4, 16, 16>;
 // the same transforms split over a cluster of 2 or 4 CTAs (smaller tiles per SM, more CTAs resident)
 using R8192x2 = Cfg<8192, 1, 32, 1, 2, 16, 32, 16>;
 using R8192x4 = Cfg<8192, 1, 32, 1, 4, 16, 32, 16>;
-using R16384x2 = Cfg<16384, 1, 32, 1, 2, 16, 4, 16, 16>;
-using R16384x4 = Cfg<16384, 1, 32, 1, 4, 16, 4, 16, 16>;
+using R16384x2 = Cfg<16384, 1, 32, 1, 2, 32, 32, 16, 1, 4>;
+using R16384x4 = Cfg<16384, 1, 32, 1, 4, 32, 32, 16, 1, 4>;
 // past the single-CTA limit: one 32768-point transform over a cluster of 2 CTAs of 16384 points each, still
 // one pass over main memory (the first exchange goes through distributed shared memory). Measured on B200
 // against the two-pass split: 627 against 713 us for 4096 transforms, 16.8 against 21.2 us for 64, and no
