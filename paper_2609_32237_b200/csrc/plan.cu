@@ -231,7 +231,7 @@ extern "C" int fft_plan_set_option(fft_plan_t p, const char* key, int64_t value)
         return B200FFT_OK;
     }
     if (std::strcmp(key, "cluster") == 0) {
-        if (p->four_step || p->n > 16384) return B200FFT_ERR_UNSUPPORTED;
+        if (p->four_step || p->n > 32768) return B200FFT_ERR_UNSUPPORTED;
         const int old = p->cluster;
         p->cluster = (int)value;
         int rc = build_single_pass(p);
