@@ -12,8 +12,10 @@ using R128 = Cfg<128, 1, 16, 16, 1, 16, 8>;
 using R64 = Cfg<64, 1, 16, 32, 1, 8, 8>;
 using R32 = Cfg<32, 1, 16, 64, 1, 4, 8>;
 using R256 = Cfg<256, 1, 32, 16, 1, 16, 16>;
-using R512 = Cfg<512, 1, 32, 8, 1, 16, 2, 16>;
-using R1024 = Cfg<1024, 1, 32, 4, 1, 16, 4, 16>;
+using R512 = Cfg<512, 1, 32, 8, 1, 16, 32>;
+using R1024 = Cfg<1024, 1, 32, 4, 1, 32, 32>;
+// for kernels that work on register pairs at both ends of the network (fused range compression)
+using R1024p = Cfg<1024, 1, 32, 4, 1, 16, 4, 16>;
 using R2048 = Cfg<2048, 1, 32, 2, 1, 16, 8, 16>;
 using R4096 = Cfg<4096, 1, 32, 1, 1, 16, 16, 16>;
 using R8192 = Cfg<8192, 1, 32, 1, 1, 16, 32, 16>;

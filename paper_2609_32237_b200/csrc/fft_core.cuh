@@ -569,6 +569,7 @@ struct Engine {
     __device__ __forceinline__ void store_first(void* out, int64_t base, int64_t ld, float scale) {
         using G = Geo<C, 1>;
         constexpr int V = G::V, r = G::r;
+        static_assert(V >= 2, "store_first writes register pairs");
         static_for<0, V / 2>([&](auto h_) {
             constexpr int v = 2 * decltype(h_)::value;
             const int c = C::template cidx<V>(t, v, rank);

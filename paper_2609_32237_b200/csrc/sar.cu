@@ -47,6 +47,8 @@ template <class C, class TOut>
 __global__ void __launch_bounds__(C::THREADS, C::MINB) sar_range_compress_kernel(const SarArgs a) {
     extern __shared__ __align__(16) float2 smem_dyn[];
     static_assert(C::W == 1, "range compression works on contiguous rows");
+    static_assert(C::P / C::radix(1) >= 2 && C::P / C::radix(C::S) >= 2,
+                  "the filter multiply and the final store work on register pairs: two butterflies per thread at both ends");
     const int g = threadIdx.x / C::T, t = threadIdx.x % C::T;
     int64_t tile = (C::CL > 1) ? (int64_t)(blockIdx.x / C::CL) : (int64_t)blockIdx.x * C::G + g;
     const bool active = tile < a.tiles;
@@ -461,7 +463,7 @@ constexpr SarEntry sar_entry() {
     else return SarEntry{C::N, T::ELEM_BYTES == 8 ? 0 : 1, C::W, C::TW_TOTAL, &launch_rcmc<C, T>, &launch_build_tw<C>};
 }
 #define SAR_PAIR(C, RANGE) sar_entry<C, StoreC64, RANGE>(), sar_entry<C, StoreC32H, RANGE>()
-static const SarEntry k_range[] = {SAR_PAIR(R1024, true), SAR_PAIR(R2048, true), SAR_PAIR(R4096, true), SAR_PAIR(R8192, true)};
+static const SarEntry k_range[] = {SAR_PAIR(R1024p, true), SAR_PAIR(R2048, true), SAR_PAIR(R4096, true), SAR_PAIR(R8192, true)};
 static const SarEntry k_rcmc[] = {SAR_PAIR(T1024, false), SAR_PAIR(T2048, false), SAR_PAIR(T4096, false)};
 
 template <size_t K>
