@@ -51,6 +51,9 @@ def test_bad_arguments_are_rejected_on_the_host(B):
     assert h.value is None
     assert L.fft_execute(None, None, None, None) == 1
     assert L.fft_plan_destroy(None) == 1
+    assert L.fft_execute_bfp(None, None, None, None, None, None) == 1
+    assert L.fft_plan_set_option(None, b"staged", 1) == 1
+    assert L.fft_execute_noalloc(4096, 1 << 20, -1, None, None, None) != 0     # beyond the fixed scratch, or null
     assert L.sar_rda_params_create(None, None) == 1
     d = B.SarRdaDesc(n_azimuth=4096, n_range=4096, carrier_hz=9.6e9, bandwidth_hz=1e8, fs_hz=1.2e8,
                      pulse_s=1e-5, prf_hz=1000.0, velocity_mps=200.0, r_center_m=1e4,
