@@ -160,6 +160,16 @@ struct Dft<32> {
     static __device__ __forceinline__ void run(float2* v) { dft_composite<32, 4, 8>(v); }
 };
 
+// Order in which the r inputs of a butterfly are fetched: the composite transforms work on the
+// subsets j = a + A b first (a fixed), so fetching subset by subset lets the arithmetic on the
+// first subset start while the rest are still in flight.
+template <int R>
+__host__ __device__ constexpr int fetch_order(int i) {
+    constexpr int A = (R == 32 || R == 16) ? 4 : (R == 8 ? 2 : 1);
+    constexpr int B = R / A;
+    return (i / B) + A * (i % B);
+}
+
 // ------------------------------------------------------------ configuration
 template <int N_, int W_, int P_, int G_, int CL_, int R1_, int R2_, int R3_ = 1, int R4_ = 1, int TW1_ = 1>
 struct Cfg {
@@ -400,8 +410,8 @@ struct Engine {
                 constexpr int v = 2 * decltype(h_)::value;
                 G g;
                 g.init(t, v, rank);
-                static_for<0, r>([&](auto j_) {
-                    constexpr int j = decltype(j_)::value;
+                static_for<0, r>([&](auto i_) {
+                    constexpr int j = WR ? decltype(i_)::value : fetch_order<r>(decltype(i_)::value);
                     float2* p2 = sm + g.template elem<j>();
                     if constexpr (WR) {
                         const float4 val = make_float4(x[j * V + v].x, x[j * V + v].y, x[j * V + v + 1].x, x[j * V + v + 1].y);
@@ -417,8 +427,8 @@ struct Engine {
         } else {
             G g;
             g.init(t, 0, rank);
-            static_for<0, r>([&](auto j_) {
-                constexpr int j = decltype(j_)::value;
+            static_for<0, r>([&](auto i_) {
+                constexpr int j = WR ? decltype(i_)::value : fetch_order<r>(decltype(i_)::value);
                 float2* p2 = sm + g.template elem<j>();
                 if constexpr (WR) {
                     if constexpr (REMOTE) st_cluster_f2(p2, (unsigned)G::template dest<j>(), x[j]);
@@ -543,8 +553,8 @@ struct Engine {
                                     // still one contiguous run per warp
             const int c = C::template cidx<1>(t, 0, rank);
             const int q = c % W, lo = c / W;
-            static_for<0, r>([&](auto j_) {
-                constexpr int j = decltype(j_)::value;
+            static_for<0, r>([&](auto i_) {
+                constexpr int j = fetch_order<r>(decltype(i_)::value);
                 const int64_t idx = (W == 1) ? base + j * G::Ls + lo : base + (int64_t)(j * G::Ls + lo) * ld + q;
                 x[j] = ST::load1(in, idx);
                 if constexpr (CONJ) x[j].y = -x[j].y;
@@ -554,8 +564,8 @@ struct Engine {
             constexpr int v = 2 * decltype(h_)::value;
             const int c = C::template cidx<V>(t, v, rank);
             const int q = c % W, lo = c / W;
-            static_for<0, r>([&](auto j_) {
-                constexpr int j = decltype(j_)::value;
+            static_for<0, r>([&](auto i_) {
+                constexpr int j = fetch_order<r>(decltype(i_)::value);
                 const int64_t idx = (W == 1) ? base + j * G::Ls + lo : base + (int64_t)(j * G::Ls + lo) * ld + q;
                 ST::load2(in, idx, x[j * V + v], x[j * V + v + 1]);
                 if constexpr (CONJ) {
