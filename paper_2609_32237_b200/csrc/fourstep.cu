@@ -56,19 +56,21 @@ __global__ void __launch_bounds__(C::THREADS, C::MINB) fourstep_pass1_kernel(con
     if (!active) return;
     using G = Geo<C, C::S>;
     constexpr int V = G::V, r = G::r, KS = C::N / r;
-    const int64_t nmask = a.n - 1;
+    // k1 < n1 <= 1024 and j2 < n2 <= 1024: the products fit 32 bits
+    const unsigned nmask = (unsigned)(a.n - 1), n2 = (unsigned)a.n2;
+    const int64_t obase = b * a.dist_out;
     static_for<0, V / 2>([&](auto h_) {
         constexpr int v = 2 * decltype(h_)::value;
         int b0, q;
         e.last_index(v, b0, q);
-        const int64_t j2 = cg * W + q;
+        const unsigned j2 = (unsigned)cg * W + q;
         static_for<0, r>([&](auto j_) {
             constexpr int j = decltype(j_)::value;
-            const int64_t k1 = j * KS + b0;
-            const int64_t m0 = (k1 * j2) & nmask;
+            const unsigned k1 = j * KS + b0;
+            const unsigned m0 = (k1 * j2) & nmask;
             const float2 w0 = cmul(__ldg(a.tw_hi + (m0 >> 10)), __ldg(a.tw_lo + (m0 & 1023)));
             const float2 w1 = cmul(w0, __ldg(a.tw_lo + k1));     // one column on: times exp(-2 pi i k1 / n), k1 < 1024
-            TOut::store2(a.out, b * a.dist_out + k1 * a.n2 + j2, cmul(e.x[j * V + v], w0), cmul(e.x[j * V + v + 1], w1));
+            TOut::store2(a.out, obase + (k1 * n2 + j2), cmul(e.x[j * V + v], w0), cmul(e.x[j * V + v + 1], w1));
         });
     });
 }
@@ -89,15 +91,16 @@ __global__ void __launch_bounds__(C::THREADS, C::MINB) fourstep_pass2_kernel(con
         using G = Geo<C, 1>;
         constexpr int V = G::V, r = G::r;
         const int64_t rowbase = b * a.dist_in + rg * W * a.n2;
+        const unsigned n2 = (unsigned)a.n2;                 // W * n2 <= 16384: offsets within the tile fit 32 bits
         static_for<0, V / 2>([&](auto h_) {
             constexpr int v = 2 * decltype(h_)::value;
             const int c = C::template cidx<V>(e.t, v, e.rank);
-            const int q = c % W, lo = c / W;
-            static_for<0, r>([&](auto j_) {
-                constexpr int j = decltype(j_)::value;
-                const int64_t idx = rowbase + (int64_t)q * a.n2 + j * G::Ls + lo;
-                e.x[j * V + v] = TIn::load1(a.in, idx);
-                e.x[j * V + v + 1] = TIn::load1(a.in, idx + a.n2);
+            const unsigned q = c % W, lo = c / W;
+            const int64_t pbase = rowbase + (q * n2 + lo);
+            static_for<0, r>([&](auto i_) {
+                constexpr int j = fetch_order<r>(decltype(i_)::value);
+                e.x[j * V + v] = TIn::load1(a.in, pbase + j * G::Ls);
+                e.x[j * V + v + 1] = TIn::load1(a.in, pbase + j * G::Ls + n2);
             });
         });
     }
@@ -108,10 +111,15 @@ __global__ void __launch_bounds__(C::THREADS, C::MINB) fourstep_pass2_kernel(con
 template <class C, bool INV, class TI, class TO, int PASS>
 cudaError_t launch_fourstep(const FourStepArgs& a, cudaStream_t st) {
     static bool done[64] = {};
-    auto kernel = (PASS == 1) ? fourstep_pass1_kernel<C, INV, TI, TO> : fourstep_pass2_kernel<C, INV, TI, TO>;
-    cudaError_t e = ensure_smem(kernel, C::SMEM_BYTES, done);
-    if (e != cudaSuccess) return e;
-    return launch_tiles<C>(kernel, a, a.tiles, st);
+    if constexpr (PASS == 1) {          // (a ternary would instantiate both kernels for every configuration)
+        cudaError_t e = ensure_smem(fourstep_pass1_kernel<C, INV, TI, TO>, C::SMEM_BYTES, done);
+        if (e != cudaSuccess) return e;
+        return launch_tiles<C>(fourstep_pass1_kernel<C, INV, TI, TO>, a, a.tiles, st);
+    } else {
+        cudaError_t e = ensure_smem(fourstep_pass2_kernel<C, INV, TI, TO>, C::SMEM_BYTES, done);
+        if (e != cudaSuccess) return e;
+        return launch_tiles<C>(fourstep_pass2_kernel<C, INV, TI, TO>, a, a.tiles, st);
+    }
 }
 
 template <class C, bool INV, class TS, int PASS>
