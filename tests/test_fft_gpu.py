@@ -297,7 +297,7 @@ def test_execute_host_pipelined_and_simple_paths():
     batch) and the plain path (small batch) both match the device-resident call."""
     import torch
     from paper_2609_32237_b200 import binding as B
-    for n, batch in ((1024, 8192), (4096, 6)):
+    for n, batch in ((1024, 8192), (4096, 6), (32768, 160)):     # the last: the cluster kernel, chunk by chunk
         x = inputs.gaussian_complex64((batch, n), 97)
         h_in = torch.from_numpy(x).pin_memory()
         h_out = torch.zeros_like(h_in).pin_memory()
@@ -515,3 +515,27 @@ def test_n32768_runs_in_one_pass_on_a_cluster_of_two():
     want = oracle.fft_rows(inputs.from_half_storage(h), FWD)
     got = half_to_c128(run_fft(to_device_half(h), n, batch, 1, n, FWD, C32H))
     assert max(worst_rel_l2(got, want)) <= TOL16
+
+
+def test_execute_host_with_fp16_storage_and_the_staged_kernel():
+    """The chunked host path on fp16 storage at n = 16384, where the persistent staged kernel is the
+    default and every chunk is one launch of it with fewer tiles than CTAs."""
+    import torch
+    from paper_2609_32237_b200 import binding as B
+    n, batch = 16384, 640
+    h = inputs.to_half_storage(inputs.gaussian_complex64((batch, n), 98))
+    h_in = torch.from_numpy(h).pin_memory()
+    h_out = torch.zeros_like(h_in).pin_memory()
+    d_in = torch.zeros(batch, n, 2, dtype=torch.float16, device="cuda")
+    d_out = torch.zeros_like(d_in)
+    plan = B.fft_plan_create(n, batch, 1, n, FWD, C32H)
+    try:
+        B.fft_execute_host(plan, h_in.data_ptr(), h_out.data_ptr(), d_in.data_ptr(), d_out.data_ptr(),
+                           torch.cuda.current_stream().cuda_stream)
+        torch.cuda.synchronize()
+    finally:
+        B.fft_plan_destroy(plan)
+    idx = inputs.sample_indices(batch, 6, 4)
+    want = oracle.fft_rows(inputs.from_half_storage(h[idx]), FWD)
+    assert max(worst_rel_l2(half_to_c128(h_out[torch.from_numpy(idx)]), want)) <= TOL16
+    assert B.tma_timeouts() == 0
