@@ -147,6 +147,67 @@ __device__ __forceinline__ void dft_composite(float2* v) {
         static_for<0, A>([&](auto d_) { constexpr int d = decltype(d_)::value; v[c + B * d] = t[d]; });
     });
 }
+// The same for two butterflies at once, handing every finished output pair (k, a_k, b_k) to `emit`
+// as soon as its last small transform is done, so that stores can leave while the rest is computed.
+template <int R, int A, int B, class F>
+__device__ __forceinline__ void dft_composite_emit2(const float2* va, const float2* vb, F&& emit) {
+    float2 ya[R], yb[R];
+    static_for<0, A>([&](auto a_) {
+        constexpr int a = decltype(a_)::value;
+        float2 ta[B], tb[B];
+        static_for<0, B>([&](auto b_) {
+            constexpr int b = decltype(b_)::value;
+            ta[b] = va[a + A * b];
+            tb[b] = vb[a + A * b];
+        });
+        Dft<B>::run(ta);
+        Dft<B>::run(tb);
+        static_for<0, B>([&](auto c_) {
+            constexpr int c = decltype(c_)::value;
+            ya[a * B + c] = mulw32<a * c * (32 / R)>(ta[c]);
+            yb[a * B + c] = mulw32<a * c * (32 / R)>(tb[c]);
+        });
+    });
+    static_for<0, B>([&](auto c_) {
+        constexpr int c = decltype(c_)::value;
+        float2 ta[A], tb[A];
+        static_for<0, A>([&](auto a_) {
+            constexpr int a = decltype(a_)::value;
+            ta[a] = ya[a * B + c];
+            tb[a] = yb[a * B + c];
+        });
+        Dft<A>::run(ta);
+        Dft<A>::run(tb);
+        static_for<0, A>([&](auto d_) {
+            constexpr int d = decltype(d_)::value;
+            emit(IntC<c + B * d>{}, ta[d], tb[d]);
+        });
+    });
+}
+template <int R, int A, int B, class F>
+__device__ __forceinline__ void dft_composite_emit1(const float2* va, F&& emit) {
+    float2 ya[R];
+    static_for<0, A>([&](auto a_) {
+        constexpr int a = decltype(a_)::value;
+        float2 ta[B];
+        static_for<0, B>([&](auto b_) { constexpr int b = decltype(b_)::value; ta[b] = va[a + A * b]; });
+        Dft<B>::run(ta);
+        static_for<0, B>([&](auto c_) { constexpr int c = decltype(c_)::value; ya[a * B + c] = mulw32<a * c * (32 / R)>(ta[c]); });
+    });
+    static_for<0, B>([&](auto c_) {
+        constexpr int c = decltype(c_)::value;
+        float2 ta[A];
+        static_for<0, A>([&](auto a_) { constexpr int a = decltype(a_)::value; ta[a] = ya[a * B + c]; });
+        Dft<A>::run(ta);
+        static_for<0, A>([&](auto d_) { constexpr int d = decltype(d_)::value; emit(IntC<c + B * d>{}, ta[d]); });
+    });
+}
+template <int R>
+struct Split;      // R = A * B as used by Dft<R>
+template <> struct Split<8> { static constexpr int A = 2, B = 4; };
+template <> struct Split<16> { static constexpr int A = 4, B = 4; };
+template <> struct Split<32> { static constexpr int A = 4, B = 8; };
+
 template <>
 struct Dft<8> {
     static __device__ __forceinline__ void run(float2* v) { dft_composite<8, 2, 4>(v); }
@@ -645,13 +706,61 @@ struct Engine {
         });
     }
 
+    // Last stage and global store in one: every output pair is stored as soon as it is final.
+    template <class ST, bool CONJ>
+    __device__ __forceinline__ void last_stage_and_store(void* out, int64_t base, int64_t ld, float scale) {
+        using G = Geo<C, S>;
+        constexpr int V = G::V, r = G::r, KS = C::N / r;
+        if constexpr (V >= 2 && (r == 8 || r == 16 || r == 32)) {
+            const bool scaled = scale != 1.0f;
+            static_for<0, V / 2>([&](auto h_) {
+                constexpr int v = 2 * decltype(h_)::value;
+                int b0, q;
+                last_index(v, b0, q);
+                float2 a[r], b[r];
+                static_for<0, r>([&](auto j_) {
+                    constexpr int j = decltype(j_)::value;
+                    a[j] = x[j * V + v];
+                    b[j] = x[j * V + v + 1];
+                });
+                dft_composite_emit2<r, Split<r>::A, Split<r>::B>(a, b, [&](auto k_, float2 pa, float2 pb) {
+                    constexpr int k = decltype(k_)::value;
+                    const int64_t idx = (W == 1) ? base + k * KS + b0 : base + (int64_t)(k * KS + b0) * ld + q;
+                    if constexpr (CONJ) {
+                        pa.y = -pa.y;
+                        pb.y = -pb.y;
+                    }
+                    if (scaled) {
+                        pa = make_float2(pa.x * scale, pa.y * scale);
+                        pb = make_float2(pb.x * scale, pb.y * scale);
+                    }
+                    ST::store2(out, idx, pa, pb);
+                });
+            });
+        } else if constexpr (V == 1 && W == 1 && (r == 8 || r == 16 || r == 32)) {
+            const bool scaled = scale != 1.0f;
+            int b0, q;
+            last_index(0, b0, q);
+            dft_composite_emit1<r, Split<r>::A, Split<r>::B>(x, [&](auto k_, float2 pa) {
+                constexpr int k = decltype(k_)::value;
+                if constexpr (CONJ) pa.y = -pa.y;
+                if (scaled) pa = make_float2(pa.x * scale, pa.y * scale);
+                ST::store1(out, base + k * KS + b0, pa);
+            });
+        } else {
+            compute<S, false>(nullptr);
+            store_last<ST, CONJ>(out, base, ld, scale);
+        }
+    }
+
     // ---- whole networks ---------------------------------------------------------------
     // registers hold stage-1 layout on entry; on exit they hold the last stage's
     // layout: x[j*V + v] = X[b0 + (N/r_S) j] for butterfly pair v (digit-reversed positions)
+    template <bool LAST_COMPUTE = true>
     __device__ __forceinline__ void dif(float2* sm, const float2* __restrict__ tw) {
         static_for<1, S + 1>([&](auto s_) {
             constexpr int s = decltype(s_)::value;
-            compute<s, false>(tw);
+            if constexpr (s < S || LAST_COMPUTE) compute<s, false>(tw);
             if constexpr (s < S) {
                 if constexpr (CL > 1 && s == 1) cluster_wait();   // pairs with the arrive in setup()
                 smem_rw<s, true>(sm);
@@ -719,8 +828,8 @@ __global__ void __launch_bounds__(C::THREADS, C::MINB) fft_kernel(const FftArgs 
                              SHARE);
     }
     e.template load_first<TIn, INV>(a.in, base, a.dist);
-    e.dif(sm, a.tw);
-    if (active) e.template store_last<TOut, INV>(a.out, base, a.dist, a.scale);
+    e.template dif<false>(sm, a.tw);
+    if (active) e.template last_stage_and_store<TOut, INV>(a.out, base, a.dist, a.scale);
 }
 
 // Builds the per-stage twiddle rows of a configuration in float64, rounds once to fp32:

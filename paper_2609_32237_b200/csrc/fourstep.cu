@@ -104,8 +104,8 @@ __global__ void __launch_bounds__(C::THREADS, C::MINB) fourstep_pass2_kernel(con
             });
         });
     }
-    e.dif(sm, a.tw);
-    if (active) e.template store_last<TOut, INV>(a.out, b * a.dist_out + rg * W, a.n1, a.scale);
+    e.template dif<false>(sm, a.tw);
+    if (active) e.template last_stage_and_store<TOut, INV>(a.out, b * a.dist_out + rg * W, a.n1, a.scale);
 }
 
 template <class C, bool INV, class TI, class TO, int PASS>
