@@ -515,9 +515,14 @@ struct Engine {
     // ---- butterflies + twiddles ----------------------------------------------------
     // DIT = false: butterfly, then multiply output k by tw[k][lo]   (stages 1..S-1)
     // DIT = true : multiply input j by tw[j][lo], then butterfly     (transposed network)
-    template <int s, bool DIT>
-    __device__ __forceinline__ void compute(const float2* __restrict__ tw) {
+    // With a sink (stages whose butterfly comes last: the DIF last stage, every DIT stage, two
+    // butterflies per thread, radix 8/16/32) the outputs are not written back to the registers:
+    // sink(v, k, a_k, b_k) receives output k of butterflies v and v + 1 as soon as it is final.
+    struct NoSink {};
+    template <int s, bool DIT, class Sink = NoSink>
+    __device__ __forceinline__ void compute(const float2* __restrict__ tw, Sink&& sink = Sink{}) {
         using G = Geo<C, s>;
+        constexpr bool SINK = !std::is_same<typename std::decay<Sink>::type, NoSink>::value;
         constexpr int V = G::V, r = G::r, Ls = G::Ls;
         constexpr bool has_tw = !G::last;
         // Rows of the stage's twiddle table that are loaded; the rest are products of loaded
@@ -583,16 +588,23 @@ struct Engine {
                     lo0 = (C::template cidx<V>(t, v, rank) / W) % Ls;
                     if constexpr (DIT) twiddle_pair(lo0, a, b);
                 }
-                Dft<r>::run(a);
-                Dft<r>::run(b);
-                if constexpr (has_tw && !DIT) twiddle_pair(lo0, a, b);
-                static_for<0, r>([&](auto j_) {
-                    constexpr int j = decltype(j_)::value;
-                    x[j * V + v] = a[j];
-                    x[j * V + v + 1] = b[j];
-                });
+                if constexpr (SINK) {
+                    static_assert((DIT || !has_tw) && (r == 8 || r == 16 || r == 32), "a sink takes finished outputs");
+                    dft_composite_emit2<r, Split<r>::A, Split<r>::B>(
+                        a, b, [&](auto k_, float2 pa, float2 pb) { sink(IntC<v>{}, k_, pa, pb); });
+                } else {
+                    Dft<r>::run(a);
+                    Dft<r>::run(b);
+                    if constexpr (has_tw && !DIT) twiddle_pair(lo0, a, b);
+                    static_for<0, r>([&](auto j_) {
+                        constexpr int j = decltype(j_)::value;
+                        x[j * V + v] = a[j];
+                        x[j * V + v + 1] = b[j];
+                    });
+                }
             });
         } else {
+            static_assert(!SINK, "sinks are for stages with two butterflies per thread");
             [[maybe_unused]] int lo0 = 0;
             if constexpr (has_tw) {
                 lo0 = (C::template cidx<1>(t, 0, rank) / W) % Ls;
@@ -706,6 +718,24 @@ struct Engine {
         });
     }
 
+    // Stage 1 of the backward network and the natural-order global store in one.
+    template <class ST, bool CONJ>
+    __device__ __forceinline__ void first_stage_dit_and_store(const float2* __restrict__ tw, void* out, int64_t base, int64_t ld,
+                                                              float scale) {
+        using G = Geo<C, 1>;
+        constexpr int V = G::V;
+        static_assert(V >= 2, "register pairs");
+        compute<1, true>(tw, [&](auto v_, auto k_, float2 pa, float2 pb) {
+            constexpr int v = decltype(v_)::value, k = decltype(k_)::value;
+            const int c = C::template cidx<V>(t, v, rank);
+            const int q = c % W, lo = c / W;
+            const int64_t idx = (W == 1) ? base + k * G::Ls + lo : base + (int64_t)(k * G::Ls + lo) * ld + q;
+            pa = make_float2(pa.x * scale, (CONJ ? -pa.y : pa.y) * scale);
+            pb = make_float2(pb.x * scale, (CONJ ? -pb.y : pb.y) * scale);
+            ST::store2(out, idx, pa, pb);
+        });
+    }
+
     // Last stage and global store in one: every output pair is stored as soon as it is final.
     template <class ST, bool CONJ>
     __device__ __forceinline__ void last_stage_and_store(void* out, int64_t base, int64_t ld, float scale) {
@@ -771,6 +801,7 @@ struct Engine {
     }
     // registers hold the last stage's layout (digit-reversed positions) on entry,
     // stage-1 layout in natural order on exit
+    template <bool LAST_COMPUTE = true>
     __device__ __forceinline__ void dit(float2* sm, const float2* __restrict__ tw) {
         static_assert(CL == 1, "the backward network is built for single-CTA tiles");
         static_for<0, S>([&](auto i_) {
@@ -778,7 +809,7 @@ struct Engine {
             // Make the thread index opaque again at every stage: otherwise the compiler keeps
             // the address arithmetic of the forward network alive for reuse here and spills.
             asm volatile("" : "+r"(t));
-            compute<s, true>(tw);
+            if constexpr (s > 1 || LAST_COMPUTE) compute<s, true>(tw);
             if constexpr (s > 1) {
                 smem_rw<s, true>(sm);
                 __syncthreads();

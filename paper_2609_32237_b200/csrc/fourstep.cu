@@ -52,27 +52,37 @@ __global__ void __launch_bounds__(C::THREADS, C::MINB) fourstep_pass1_kernel(con
     Engine<C> e;
     e.setup(t);
     e.template load_first<TIn, INV>(a.in, b * a.dist_in + cg * W, a.n2);
-    e.dif(sm, a.tw);
+    e.template dif<false>(sm, a.tw);
     if (!active) return;
     using G = Geo<C, C::S>;
     constexpr int V = G::V, r = G::r, KS = C::N / r;
+    static_assert(V >= 2, "register pairs");
     // k1 < n1 <= 1024 and j2 < n2 <= 1024: the products fit 32 bits
     const unsigned nmask = (unsigned)(a.n - 1), n2 = (unsigned)a.n2;
     const int64_t obase = b * a.dist_out;
-    static_for<0, V / 2>([&](auto h_) {
-        constexpr int v = 2 * decltype(h_)::value;
+    auto twiddle_and_store = [&](auto v_, auto j_, float2 pa, float2 pb) {
+        constexpr int v = decltype(v_)::value, j = decltype(j_)::value;
         int b0, q;
         e.last_index(v, b0, q);
         const unsigned j2 = (unsigned)cg * W + q;
-        static_for<0, r>([&](auto j_) {
-            constexpr int j = decltype(j_)::value;
-            const unsigned k1 = j * KS + b0;
-            const unsigned m0 = (k1 * j2) & nmask;
-            const float2 w0 = cmul(__ldg(a.tw_hi + (m0 >> 10)), __ldg(a.tw_lo + (m0 & 1023)));
-            const float2 w1 = cmul(w0, __ldg(a.tw_lo + k1));     // one column on: times exp(-2 pi i k1 / n), k1 < 1024
-            TOut::store2(a.out, obase + (k1 * n2 + j2), cmul(e.x[j * V + v], w0), cmul(e.x[j * V + v + 1], w1));
+        const unsigned k1 = j * KS + b0;
+        const unsigned m0 = (k1 * j2) & nmask;
+        const float2 w0 = cmul(__ldg(a.tw_hi + (m0 >> 10)), __ldg(a.tw_lo + (m0 & 1023)));
+        const float2 w1 = cmul(w0, __ldg(a.tw_lo + k1));     // one column on: times exp(-2 pi i k1 / n), k1 < 1024
+        TOut::store2(a.out, obase + (k1 * n2 + j2), cmul(pa, w0), cmul(pb, w1));
+    };
+    if constexpr (r == 8 || r == 16 || r == 32) {
+        e.template compute<C::S, false>(nullptr, twiddle_and_store);      // outputs leave as they complete
+    } else {
+        e.template compute<C::S, false>(nullptr);
+        static_for<0, V / 2>([&](auto h_) {
+            constexpr int v = 2 * decltype(h_)::value;
+            static_for<0, r>([&](auto j_) {
+                constexpr int j = decltype(j_)::value;
+                twiddle_and_store(IntC<v>{}, j_, e.x[j * V + v], e.x[j * V + v + 1]);
+            });
         });
-    });
+    }
 }
 
 template <class C, bool INV, class TIn, class TOut>

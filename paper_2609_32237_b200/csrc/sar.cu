@@ -77,8 +77,8 @@ __global__ void __launch_bounds__(C::THREADS, C::MINB) sar_range_compress_kernel
             });
         });
     }
-    e.dit(sm, a.tw);
-    if (active) e.template store_first<TOut, true>(a.out, base, a.ld, 1.0f);
+    e.template dit<false>(sm, a.tw);
+    if (active) e.template first_stage_dit_and_store<TOut, true>(a.tw, a.out, base, a.ld, 1.0f);
 }
 
 // ---------------------------------------------------------------- step 2
