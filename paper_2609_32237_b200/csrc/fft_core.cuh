@@ -203,7 +203,7 @@ __device__ __forceinline__ void dft_composite_emit1(const float2* va, F&& emit) 
     });
 }
 template <int R>
-struct Split;      // R = A * B as used by Dft<R>
+struct Split { static constexpr int A = 1, B = R; };      // R = A * B as used by Dft<R> (8, 16, 32 below)
 template <> struct Split<8> { static constexpr int A = 2, B = 4; };
 template <> struct Split<16> { static constexpr int A = 4, B = 4; };
 template <> struct Split<32> { static constexpr int A = 4, B = 8; };
@@ -615,6 +615,61 @@ struct Engine {
         }
     }
 
+    // Butterfly, twiddle and shared-memory write of a stage s < S in one: output k is multiplied by its
+    // twiddle and written as soon as its last small transform is done, so the write phase overlaps the
+    // arithmetic. For stages whose twiddle rows are all loaded (any order of k), local shared memory.
+    template <int s>
+    __host__ __device__ static constexpr bool fused_write_ok() {
+        constexpr int r = C::radix(s);
+        constexpr int M = (s == 1 && W == 1 && r > C::TW1_LOADS) ? C::TW1_LOADS : r - 1;
+        return s < S && M == r - 1 && !(CL > 1 && s == 1) && (r == 8 || r == 16 || r == 32);
+    }
+    template <int s>
+    __device__ __forceinline__ void compute_and_write(float2* sm, const float2* __restrict__ tw) {
+        using G = Geo<C, s>;
+        constexpr int V = G::V, r = G::r, Ls = G::Ls;
+        if constexpr (V >= 2) {
+            static_for<0, V / 2>([&](auto h_) {
+                constexpr int v = 2 * decltype(h_)::value;
+                float2 a[r], b[r];
+                static_for<0, r>([&](auto j_) {
+                    constexpr int j = decltype(j_)::value;
+                    a[j] = x[j * V + v];
+                    b[j] = x[j * V + v + 1];
+                });
+                const int lo0 = (C::template cidx<V>(t, v, rank) / W) % Ls;
+                const float2* row = tw + C::tw_off(s) + lo0;
+                G g;
+                g.init(t, v, rank);
+                dft_composite_emit2<r, Split<r>::A, Split<r>::B>(a, b, [&](auto k_, float2 pa, float2 pb) {
+                    constexpr int k = decltype(k_)::value;
+                    if constexpr (k > 0) {
+                        if constexpr (W == 1) {
+                            const float4 w = __ldg(reinterpret_cast<const float4*>(row + (k - 1) * Ls));
+                            pa = cmul(pa, make_float2(w.x, w.y));
+                            pb = cmul(pb, make_float2(w.z, w.w));
+                        } else {
+                            const float2 w = __ldg(row + (k - 1) * Ls);
+                            pa = cmul(pa, w);
+                            pb = cmul(pb, w);
+                        }
+                    }
+                    *reinterpret_cast<float4*>(sm + g.template elem<k>()) = make_float4(pa.x, pa.y, pb.x, pb.y);
+                });
+            });
+        } else {
+            const int lo0 = (C::template cidx<1>(t, 0, rank) / W) % Ls;
+            const float2* row = tw + C::tw_off(s) + lo0;
+            G g;
+            g.init(t, 0, rank);
+            dft_composite_emit1<r, Split<r>::A, Split<r>::B>(x, [&](auto k_, float2 pa) {
+                constexpr int k = decltype(k_)::value;
+                if constexpr (k > 0) pa = cmul(pa, __ldg(row + (k - 1) * Ls));
+                sm[g.template elem<k>()] = pa;
+            });
+        }
+    }
+
     // ---- global access with the stage-1 mapping (natural-order positions) --------------
     // position of register (j, v): p = j * L1 + lo; rows: index base + p (+1 for v odd);
     // columns: index base + p * ld + q.
@@ -790,12 +845,18 @@ struct Engine {
     __device__ __forceinline__ void dif(float2* sm, const float2* __restrict__ tw) {
         static_for<1, S + 1>([&](auto s_) {
             constexpr int s = decltype(s_)::value;
-            if constexpr (s < S || LAST_COMPUTE) compute<s, false>(tw);
-            if constexpr (s < S) {
-                if constexpr (CL > 1 && s == 1) cluster_wait();   // pairs with the arrive in setup()
-                smem_rw<s, true>(sm);
-                exchange_barrier<(CL > 1 && s == 1)>();
+            if constexpr (fused_write_ok<s>()) {
+                compute_and_write<s>(sm, tw);
+                __syncthreads();
                 smem_rw<s + 1, false>(sm);
+            } else {
+                if constexpr (s < S || LAST_COMPUTE) compute<s, false>(tw);
+                if constexpr (s < S) {
+                    if constexpr (CL > 1 && s == 1) cluster_wait();   // pairs with the arrive in setup()
+                    smem_rw<s, true>(sm);
+                    exchange_barrier<(CL > 1 && s == 1)>();
+                    smem_rw<s + 1, false>(sm);
+                }
             }
         });
     }
