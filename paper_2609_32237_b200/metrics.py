@@ -13,7 +13,7 @@ BYTES_PER_POINT = {0: 16, 1: 8}        # storage dtype -> bytes in + bytes out p
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures
 # summarised under profiles/ (None until a capture exists for that kernel)
-NCU_TRAFFIC_BYTES = {"fft_rows_4096_c64": 2096803000}
+NCU_TRAFFIC_BYTES = {"fft_rows_4096_c64": 2095526000}
 
 
 def fft_flops(n: int, batch: int = 1) -> float:
