@@ -31,7 +31,7 @@ using R16384x2 = Cfg<16384, 1, 32, 1, 2, 32, 32, 16, 1, 4>;
 using R16384x4 = Cfg<16384, 1, 32, 1, 4, 32, 32, 16, 1, 4>;
 // past the single-CTA limit: one 32768-point transform over a cluster of 2 CTAs of 16384 points each, still
 // one pass over main memory (the first exchange goes through distributed shared memory). Measured on B200
-// against the two-pass split: 627 against 713 us for 4096 transforms, 16.8 against 21.2 us for 64, and no
+// against the two-pass split: 609 against 706 us for 4096 transforms, 16.8 against 21.2 us for 64, and no
 // workspace (32 x 32 x 32: the last stage has one butterfly per thread and stores 64 bits per lane; the
 // four-stage 32 x 4 x 16 x 16 took 693 us). The same with 4 CTAs at 65536 points (32 x 8 x 16 x 16) and 8 CTAs
 // at 131072 (32 x 16 x 16 x 16) is correct but slower than two passes (876 against 745 us, 1134 against 831 us)
