@@ -136,15 +136,7 @@ int tma_timeouts() {
 static const KernelEntry k_cols[] = {
     B200FFT_ENTRIES_STD(T256),  B200FFT_ENTRIES_STD(T512),  B200FFT_ENTRIES_STD(T1024),
     B200FFT_ENTRIES_STD(T2048), B200FFT_ENTRIES_STD(T4096), B200FFT_ENTRIES_STD(T8192),
-    B200FFT_ENTRIES_STD(T2048x2), B200FFT_ENTRIES_STD(T4096x2), B200FFT_ENTRIES_STD(T4096x4),
-    B200FFT_ENTRIES_STD(T8192x2),
 };
-
-// Wide tiles (16 columns: whole 128-byte row segments; 8 at n = 1024) for the shorter transforms, taken
-// by default when the batch is a multiple of the tile width. Measured on B200 for a 128 MiB matrix,
-// complex64 / fp16 storage: n = 256: 64 -> 54 us / 58 -> 37 us; n = 512: 70 -> 62 us; n = 1024: 74 -> 68 us /
-// 74 -> 55 us. At n = 2048 an 8-column tile fills the SM and gains nothing (80 us either way).
-static const KernelEntry k_cols_wide[] = {B200FFT_ENTRIES_STD(F256), B200FFT_ENTRIES_STD(F512), B200FFT_ENTRIES_STD(F1024)};
 
 static int default_cluster(int n) { return 1; }
 
@@ -154,14 +146,22 @@ const KernelEntry* find_cols_kernel(int n, bool inverse, int in_dtype, int out_d
             if (e.n == n && e.inverse == inverse && e.in_dtype == in_dtype && e.out_dtype == out_dtype) return &e;
         return nullptr;
     }
-    if (cl == 1019) {                                 // wide tiles
-        for (const KernelEntry& e : k_cols_wide)
-            if (e.n == n && e.inverse == inverse && e.in_dtype == in_dtype && e.out_dtype == out_dtype) return &e;
+    const EntryList more = cols_entries_more();
+    if (cl == 1019) {                                 // wide tiles (their entries carry w > 4)
+        for (int i = 0; i < more.count; ++i) {
+            const KernelEntry& e = more.first[i];
+            if (e.w > 4 && e.n == n && e.inverse == inverse && e.in_dtype == in_dtype && e.out_dtype == out_dtype) return &e;
+        }
         return nullptr;
     }
     if (cl == 0) cl = default_cluster(n);
     for (const KernelEntry& e : k_cols)
         if (e.n == n && e.cl == cl && e.inverse == inverse && e.in_dtype == in_dtype && e.out_dtype == out_dtype) return &e;
+    for (int i = 0; i < more.count; ++i) {
+        const KernelEntry& e = more.first[i];
+        if (e.w <= 4 && e.n == n && e.cl == cl && e.inverse == inverse && e.in_dtype == in_dtype && e.out_dtype == out_dtype)
+            return &e;
+    }
     return nullptr;
 }
 

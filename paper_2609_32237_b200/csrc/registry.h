@@ -93,6 +93,16 @@ struct BfpEntry {
 };
 const BfpEntry* find_bfp_kernel(int n, bool inverse);
 
+// The kernel tables are spread over several translation units so that they compile in parallel.
+struct EntryList {
+    const KernelEntry* first;
+    int count;
+};
+EntryList rows_entries_small();     // N = 32 .. 2048
+EntryList rows_entries_large();     // N = 4096 .. 16384 and the alternative factorisations
+EntryList rows_entries_cluster();   // transforms shared by a cluster of CTAs
+EntryList cols_entries_more();      // column tiles on clusters, wide column tiles
+
 // cl: CTAs per tile (cluster size); 0 picks the default variant for that size
 const KernelEntry* find_rows_kernel(int n, bool inverse, int in_dtype, int out_dtype, int cl = 0,
                                     int64_t batch = (int64_t)1 << 40);
