@@ -137,8 +137,8 @@ __global__ void __launch_bounds__(C::THREADS, CTAS_PER_SM) fft_rows_staged_kerne
 template <class C, bool INV, class TI, class TO, int CPS>
 cudaError_t launch_staged(const FftArgs& a, cudaStream_t st) {
     using L = Staged<C, TI, CPS>;
-    // the copy engine wants 16-byte aligned sources (the plan checks that already); anything else takes the plain kernel
-    if ((reinterpret_cast<uintptr_t>(a.in) & 15) || ((a.dist * L::EB) & 15)) return launch_fft<C, INV, TI, TO>(a, st);
+    // the copy engine wants 16-byte aligned sources; the plan has checked that already
+    if ((reinterpret_cast<uintptr_t>(a.in) & 15) || ((a.dist * L::EB) & 15)) return cudaErrorMisalignedAddress;
     static bool done[64] = {};
     static int sms[64] = {};
     cudaError_t e = ensure_smem(fft_rows_staged_kernel<C, INV, TI, TO, CPS>, L::SMEM_BYTES, done);
