@@ -147,10 +147,18 @@ const KernelEntry* find_cols_kernel(int n, bool inverse, int in_dtype, int out_d
         return nullptr;
     }
     const EntryList more = cols_entries_more();
+    if (cl == 1023) {                                 // wider tiles on a cluster of two CTAs
+        for (int i = 0; i < more.count; ++i) {
+            const KernelEntry& e = more.first[i];
+            if (e.cl == 2 && e.w * e.n == 32768 && e.n == n && e.inverse == inverse && e.in_dtype == in_dtype && e.out_dtype == out_dtype)
+                return &e;
+        }
+        return nullptr;
+    }
     if (cl == 1019) {                                 // wide tiles (their entries carry w > 4)
         for (int i = 0; i < more.count; ++i) {
             const KernelEntry& e = more.first[i];
-            if (e.w > 4 && e.n == n && e.inverse == inverse && e.in_dtype == in_dtype && e.out_dtype == out_dtype) return &e;
+            if (e.w > 4 && e.cl == 1 && e.n == n && e.inverse == inverse && e.in_dtype == in_dtype && e.out_dtype == out_dtype) return &e;
         }
         return nullptr;
     }
@@ -159,7 +167,7 @@ const KernelEntry* find_cols_kernel(int n, bool inverse, int in_dtype, int out_d
         if (e.n == n && e.cl == cl && e.inverse == inverse && e.in_dtype == in_dtype && e.out_dtype == out_dtype) return &e;
     for (int i = 0; i < more.count; ++i) {
         const KernelEntry& e = more.first[i];
-        if (e.w <= 4 && e.n == n && e.cl == cl && e.inverse == inverse && e.in_dtype == in_dtype && e.out_dtype == out_dtype)
+        if (e.w <= 4 && e.w * e.n != 32768 && e.n == n && e.cl == cl && e.inverse == inverse && e.in_dtype == in_dtype && e.out_dtype == out_dtype)
             return &e;
     }
     return nullptr;

@@ -58,9 +58,13 @@ static int build_single_pass(b200fft_plan_s* p) {
         if (p->staged == 1 || (p->staged == -1 && by_default)) cl = 1017;
     }
     const KernelEntry* k = nullptr;
-    if (p->layout == LAYOUT_COLS && cl == 0) {          // wide tiles where they exist and divide the batch
-        k = find_cols_kernel((int)p->n, inv, p->dtype, p->dtype, 1019);
+    if (p->layout == LAYOUT_COLS && cl == 0) {          // wide tiles where they exist and divide the batch:
+        k = find_cols_kernel((int)p->n, inv, p->dtype, p->dtype, 1019);       // 16 columns for n <= 1024
         if (k && p->batch % k->w) k = nullptr;
+        if (!k) {                                                              // a cluster of two CTAs for n >= 4096
+            k = find_cols_kernel((int)p->n, inv, p->dtype, p->dtype, 1023);
+            if (k && p->batch % k->w) k = nullptr;
+        }
     }
     if (!k)
         k = (p->layout == LAYOUT_ROWS) ? find_rows_kernel((int)p->n, inv, p->dtype, p->dtype, cl, p->batch)

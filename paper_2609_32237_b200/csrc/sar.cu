@@ -523,9 +523,15 @@ extern "C" int sar_rda_params_create(sar_rda_params_t* params, const sar_rda_des
     p->d = *d;
     const int na = (int)d->n_azimuth, nr = (int)d->n_range, dt = d->intermediate_dtype;
     p->range = find(k_range, nr, dt);
-    p->azfft = find_cols_kernel(na, false, dt, dt);
+    // column tiles: the wider tile on a cluster of two CTAs where it exists and divides the range bins
+    auto cols_kernel = [&](bool inverse, int dtype) {
+        const KernelEntry* k = find_cols_kernel(na, inverse, dtype, dtype, 1023);
+        if (k && nr % k->w == 0) return k;
+        return find_cols_kernel(na, inverse, dtype, dtype);
+    };
+    p->azfft = cols_kernel(false, dt);
     p->rcmc = find(k_rcmc, na, dt);
-    p->azifft = find_cols_kernel(na, true, B200FFT_C64, B200FFT_C64);
+    p->azifft = cols_kernel(true, B200FFT_C64);
     {   // the row pass stages COLS + HALO samples: the shift may grow by at most HALO - 16 bins over COLS bins
         const double aa = wavelength * d->prf_hz / (4.0 * d->velocity_mps), u = aa * aa, sq = sqrt(1.0 - u);
         const double gmax = u / ((1.0 + sq) * sq);

@@ -541,3 +541,25 @@ def test_execute_host_with_fp16_storage_and_the_staged_kernel():
     want = oracle.fft_rows(inputs.from_half_storage(h[idx]), FWD)
     assert max(worst_rel_l2(half_to_c128(h_out[torch.from_numpy(idx)]), want)) <= TOL16
     assert B.tma_timeouts() == 0
+
+
+@pytest.mark.parametrize("n,cols,ld", [(4096, 24, 26), (4096, 8, 8), (8192, 12, 12), (8192, 4, 6)])
+def test_columns_wider_tiles_on_a_cluster_by_default(n, cols, ld):
+    """n = 4096 with a batch that is a multiple of 8, n = 8192 with a multiple of 4: the default is
+    a tile twice as wide shared by a cluster of two CTAs (64- resp. 32-byte row segments). Checked
+    against the oracle and the single-CTA tile (option cluster = 1), both directions and storage
+    types, padding untouched."""
+    m = inputs.uniform_complex64((n, ld), 63)
+    for direction in (FWD, INV):
+        want = oracle.fft_cols(m[:, :cols].astype(np.complex128), direction)
+        got = run_fft(to_device_c64(m), n, cols, ld, 1, direction, C64).cpu().numpy()
+        narrow = run_fft(to_device_c64(m), n, cols, ld, 1, direction, C64, options={"cluster": 1}).cpu().numpy()
+        per_col = np.linalg.norm(got[:, :cols] - want, axis=0) / np.linalg.norm(want, axis=0)
+        assert per_col.max() <= TOL32
+        assert rel_l2(got[:, :cols], narrow[:, :cols]) <= 1e-6
+        assert np.all(got[:, cols:] == 0)
+    if ld % 4 == 0:                                     # fp16 storage wants rows that are multiples of 16 bytes
+        h = inputs.to_half_storage(m)
+        want = oracle.fft_cols(inputs.from_half_storage(h)[:, :cols], FWD)
+        got = half_to_c128(run_fft(to_device_half(h), n, cols, ld, 1, FWD, C32H))
+        assert rel_l2(got[:, :cols], want) <= TOL16
