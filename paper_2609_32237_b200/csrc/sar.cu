@@ -523,11 +523,15 @@ extern "C" int sar_rda_params_create(sar_rda_params_t* params, const sar_rda_des
     p->d = *d;
     const int na = (int)d->n_azimuth, nr = (int)d->n_range, dt = d->intermediate_dtype;
     p->range = find(k_range, nr, dt);
-    // column tiles: the wider tile on a cluster of two CTAs where it exists and divides the range bins
+    // Column tiles. With fp16 intermediates the wider tile on a cluster of two CTAs (32-byte instead of 16-byte
+    // row segments at n_azimuth = 4096: 84 -> 77 us); with complex64 the 4-column tile measured faster inside the
+    // chain (85 against 88 us per pass), where part of the image still sits in L2.
     auto cols_kernel = [&](bool inverse, int dtype) {
-        const KernelEntry* k = find_cols_kernel(na, inverse, dtype, dtype, 1023);
-        if (k && nr % k->w == 0) return k;
-        return find_cols_kernel(na, inverse, dtype, dtype);
+        if (dtype == B200FFT_C32H) {
+            const KernelEntry* k = find_cols_kernel(na, inverse, dtype, dtype, 1023);
+            if (k && nr % k->w == 0) return k;
+        }
+        return find_cols_kernel(na, inverse, dtype, dtype, 1);
     };
     p->azfft = cols_kernel(false, dt);
     p->rcmc = find(k_rcmc, na, dt);
