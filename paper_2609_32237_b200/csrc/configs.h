@@ -63,5 +63,6 @@ using T8192x2 = Cfg<8192, 2, 32, 1, 2, 16, 32, 16>;
 // wider tiles shared by a cluster of two CTAs (16384 points each): 64-byte row segments at n = 4096, 32-byte at 8192
 using T4096w8x2 = Cfg<4096, 8, 32, 1, 2, 16, 16, 16>;
 using T8192w4x2 = Cfg<8192, 4, 32, 1, 2, 16, 32, 16>;
+using T2048w16x2 = Cfg<2048, 16, 32, 1, 2, 16, 8, 16>;
 
 }  // namespace b200fft

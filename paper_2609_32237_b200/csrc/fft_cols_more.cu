@@ -11,7 +11,7 @@ namespace b200fft {
 static const KernelEntry k_cols_more[] = {
     B200FFT_ENTRIES_STD(T2048x2), B200FFT_ENTRIES_STD(T4096x2), B200FFT_ENTRIES_STD(T4096x4), B200FFT_ENTRIES_STD(T8192x2),
     B200FFT_ENTRIES_STD(F256),    B200FFT_ENTRIES_STD(F512),    B200FFT_ENTRIES_STD(F1024),
-    B200FFT_ENTRIES_STD(T4096w8x2), B200FFT_ENTRIES_STD(T8192w4x2),
+    B200FFT_ENTRIES_STD(T4096w8x2), B200FFT_ENTRIES_STD(T8192w4x2), B200FFT_ENTRIES_STD(T2048w16x2),
 };
 
 EntryList cols_entries_more() { return EntryList{k_cols_more, (int)(sizeof(k_cols_more) / sizeof(k_cols_more[0]))}; }

@@ -543,7 +543,7 @@ def test_execute_host_with_fp16_storage_and_the_staged_kernel():
     assert B.tma_timeouts() == 0
 
 
-@pytest.mark.parametrize("n,cols,ld", [(4096, 24, 26), (4096, 8, 8), (8192, 12, 12), (8192, 4, 6)])
+@pytest.mark.parametrize("n,cols,ld", [(4096, 24, 26), (4096, 8, 8), (8192, 12, 12), (8192, 4, 6), (2048, 32, 36)])
 def test_columns_wider_tiles_on_a_cluster_by_default(n, cols, ld):
     """n = 4096 with a batch that is a multiple of 8, n = 8192 with a multiple of 4: the default is
     a tile twice as wide shared by a cluster of two CTAs (64- resp. 32-byte row segments). Checked
