@@ -134,6 +134,7 @@ int tma_timeouts() {
 }
 
 static const KernelEntry k_cols[] = {
+    B200FFT_ENTRIES_STD(T64),   B200FFT_ENTRIES_STD(T128),
     B200FFT_ENTRIES_STD(T256),  B200FFT_ENTRIES_STD(T512),  B200FFT_ENTRIES_STD(T1024),
     B200FFT_ENTRIES_STD(T2048), B200FFT_ENTRIES_STD(T4096), B200FFT_ENTRIES_STD(T8192),
 };

@@ -10,6 +10,7 @@ namespace b200fft {
 // 74 -> 55 us. At n = 2048 an 8-column tile fills the SM and gains nothing (80 us either way).
 static const KernelEntry k_cols_more[] = {
     B200FFT_ENTRIES_STD(T2048x2), B200FFT_ENTRIES_STD(T4096x2), B200FFT_ENTRIES_STD(T4096x4), B200FFT_ENTRIES_STD(T8192x2),
+    B200FFT_ENTRIES_STD(F64),     B200FFT_ENTRIES_STD(F128),
     B200FFT_ENTRIES_STD(F256),    B200FFT_ENTRIES_STD(F512),    B200FFT_ENTRIES_STD(F1024),
     B200FFT_ENTRIES_STD(T4096w8x2), B200FFT_ENTRIES_STD(T8192w4x2), B200FFT_ENTRIES_STD(T2048w16x2),
 };

@@ -470,7 +470,8 @@ def test_columns_via_transpose(n, cols, ld):
         B.fft_plan_destroy(rows_plan)
 
 
-@pytest.mark.parametrize("n,cols,ld", [(256, 32, 40), (512, 16, 16), (1024, 24, 24), (1024, 40, 48)])
+@pytest.mark.parametrize("n,cols,ld", [(256, 32, 40), (512, 16, 16), (1024, 24, 24), (1024, 40, 48), (64, 48, 52),
+                                       (128, 16, 16), (64, 20, 20), (128, 4, 4)])
 def test_columns_wide_tiles_by_default(n, cols, ld):
     """Short column transforms whose batch is a multiple of the wide tile (16 columns, 8 at
     n = 1024) take it by default: checked against the oracle and the narrow-tile kernel
