@@ -518,6 +518,11 @@ def test_n32768_runs_in_one_pass_on_a_cluster_of_two():
     want = oracle.fft_rows(inputs.from_half_storage(h), FWD)
     got = half_to_c128(run_fft(to_device_half(h), n, batch, 1, n, FWD, C32H))
     assert max(worst_rel_l2(got, want)) <= TOL16
+    # in place: both CTAs of a cluster have read their inputs before either stores (cluster barrier)
+    xc = np.ascontiguousarray(x[:, :n])
+    inplace = run_fft(to_device_c64(xc), n, batch, 1, n, FWD, C64, inplace=True).cpu().numpy()
+    outplace = run_fft(to_device_c64(xc), n, batch, 1, n, FWD, C64).cpu().numpy()
+    assert np.array_equal(inplace.view(np.uint64), outplace.view(np.uint64))
 
 
 def test_execute_host_with_fp16_storage_and_the_staged_kernel():
