@@ -107,7 +107,13 @@ int fft_plan_destroy(fft_plan_t plan);
  * "cluster" value c (1, 2 or 4; 0 = the default for that size) picks the
  * variant of a single-pass plan in which c CTAs of one thread-block cluster
  * share a tile through distributed shared memory; B200FFT_ERR_UNSUPPORTED if
- * that variant is not compiled for the plan's size. Key "prefetch" value d
+ * that variant is not compiled for the plan's size. (Defaults: rows of
+ * n = 16384 / 8192 with at most 32 / 16 transforms, and rows of n = 32768, are
+ * split over clusters; columns plans take the widest tile whose width divides
+ * the batch: 16 columns for n <= 512, 8 for n = 1024, and for n >= 2048 a tile
+ * of 32768 / n columns shared by a cluster of two CTAs, except complex64 at
+ * n = 2048; value 1 forces the single-CTA 4-column tile, 2 columns at 8192.)
+ * Key "prefetch" value d
  * makes each CTA of a rows plan ask L2 for the input of the transform d tiles
  * ahead (0 = off, -1 = the default: one wave ahead for n = 16384). Key "tma"
  * value 1 makes a complex64 columns plan (n = 1024, 2048, 4096) stage its tiles
