@@ -106,18 +106,82 @@ def single_target_xband():
     return sc, p, raw, rc, img
 
 
+def _ridge(S, k, n_t):
+    """Energy centroid of the range-Doppler spectrum of one target along range, Doppler bin k."""
+    cols = np.arange(n_t - 12, n_t + 20)
+    prof = np.abs(S[k, cols]) ** 2
+    return (prof * cols).sum() / prof.sum()
+
+
 def test_migration_formula_follows_the_simulated_trajectory(single_target_xband):
     """The simulator moves the echo along sqrt(R^2 + v^2 eta^2); in the
-    range-Doppler domain its ridge must sit at n_t + dn(k, n_t)."""
+    range-Doppler domain its ridge must sit at n_t + dn(k, n_t). The Doppler
+    bins reach to 244 Hz of the 267 Hz half band, where the ridge has moved by
+    a bin and a half, so a missing or mis-scaled migration term fails."""
     sc, p, raw, rc, img = single_target_xband
     a_t, n_t = sc.targets[0]
     assert abs(abs(rc[a_t, n_t]) - 1200) < 1e-6          # on-grid at closest approach
     S = oracle.sar_azimuth_fft(p, rc)
-    cols = np.arange(n_t - 12, n_t + 20)
-    for k in (0, 40, 120, 200, 4096 - 200, 4096 - 60):   # inside the 533 Hz Doppler band
-        prof = np.abs(S[k, cols]) ** 2
-        centroid = (prof * cols).sum() / prof.sum()
-        assert abs(centroid - (n_t + oracle.sar_migration_bins(p, k, n_t))) < 0.12
+    for k in (0, 40, 120, 200, 600, 1000, 4096 - 1000, 4096 - 600, 4096 - 200, 4096 - 60):
+        assert abs(_ridge(S, k, n_t) - (n_t + oracle.sar_migration_bins(p, k, n_t))) < 0.05
+    # the ridge itself, with no formula involved: it has left the target's bin by more than a bin
+    assert _ridge(S, 1000, n_t) - _ridge(S, 0, n_t) > 1.0
+    assert _ridge(S, 4096 - 1000, n_t) - _ridge(S, 0, n_t) > 1.0
+    assert 0.4 < _ridge(S, 600, n_t) - _ridge(S, 0, n_t) < 0.7
+    # a formula that returned no migration would miss the ridge by far more than the tolerance
+    assert abs(_ridge(S, 1000, n_t) - n_t) > 1.0
+
+
+def test_interpolator_hand_values_at_half_a_sample():
+    """mu = 1/2: sinc(1/2 - j) = (-1)^j / (pi (1/2 - j)), so the eight taps j = -3 .. 4 are
+    proportional to -1/7, 1/5, -1/3, 1, 1, -1/3, 1/5, -1/7 and sum to one."""
+    pattern = np.array([-1 / 7, 1 / 5, -1 / 3, 1.0, 1.0, -1 / 3, 1 / 5, -1 / 7])
+    np.testing.assert_allclose(oracle.sar_interp_weights(0.5), pattern / pattern.sum(), atol=1e-15)
+    # any fraction, against the library's sinc
+    for mu in (0.0, 0.125, 0.3, 0.77):
+        w = np.sinc(mu - np.arange(-3, 5))
+        np.testing.assert_allclose(oracle.sar_interp_weights(mu), w / w.sum(), atol=1e-15)
+
+
+@pytest.mark.parametrize("band", ["x", "l"])
+def test_rcmc_of_an_impulse_row_lays_out_the_taps_in_order(band):
+    """A row that is delta[n - n1] comes out as S'[k, n] = w_j(mu(k, n)) at n = n1 - i0 - j: the
+    eight weights in REVERSED tap order around n1 - i0 (tap j = 4 first), nothing elsewhere. This
+    fixes the tap orientation and the index convention n + i0 + j exactly; on the L-band scene the
+    integer shift is over a hundred bins."""
+    if band == "x":
+        sc = inputs.x_band_scene(n_azimuth=64, n_range=2048, n_targets=0)
+        ks, n1 = (0, 9, 17, 31, 33, 50), 1000
+    else:
+        sc = inputs.l_band_scene(n_azimuth=64, n_range=2048, targets=[])
+        ks, n1 = (0, 5, 22, 31, 32, 40), 1300
+    p = oracle.sar_params(sc)
+    S = np.zeros((64, 2048), dtype=np.complex128)
+    S[:, n1] = 1.0 + 0.5j
+    out = oracle.sar_rcmc(p, S)
+    lam, dr = sc.wavelength_m, sc.range_bin_m
+    biggest = 0
+    for k in ks:
+        f = (k if k < 32 else k - 64) * sc.prf_hz / 64
+        d = math.sqrt(1.0 - (lam * f / (2.0 * sc.velocity_mps)) ** 2)
+        want = np.zeros(2048, dtype=np.complex128)
+        for n in range(2048):
+            dn = (sc.r_center_m + (n - 1024) * dr) * (1.0 / d - 1.0) / dr
+            i0 = math.floor(dn)
+            j = n1 - n - i0
+            if -3 <= j <= 4:
+                w = np.sinc((dn - i0) - np.arange(-3, 5))
+                want[n] = (1.0 + 0.5j) * w[j + 3] / w.sum()
+                biggest = max(biggest, i0)
+        assert np.count_nonzero(want) == 8
+        np.testing.assert_allclose(out[k], want, atol=1e-9)
+        if k == 0:
+            assert out[k, n1] == 1.0 + 0.5j                      # no migration at zero Doppler
+        else:
+            # mirrored taps would swap the two unequal neighbours of the main tap
+            nz = np.nonzero(want)[0]
+            assert abs(abs(want[nz[3]]) - abs(want[nz[4]])) > 1e-3 or abs(abs(want[nz[2]]) - abs(want[nz[5]])) > 1e-4
+    assert biggest >= (100 if band == "l" else 5)
 
 
 def test_target_focuses_at_its_cell_with_textbook_quality(single_target_xband):

@@ -137,6 +137,32 @@ def test_config4_full_scene(dtype, tol, fused, full_scene):
 
 
 @pytest.fixture(scope="module")
+def l_band_case():
+    """The paper's worked L-band scene (wavelength 0.24 m, PRF 500 Hz, 8 m antenna, 20 km) on a
+    4096 x 2048 frame with noise: the migration correction shifts rows by up to about 190 bins
+    at the edge of the Doppler spectrum, so the moving row windows and their zero fill at the
+    row ends run with large shifts."""
+    sc = inputs.l_band_scene(n_azimuth=4096, n_range=2048, targets=[(2048, 1024), (1500, 800), (2600, 1390)])
+    sc.noise_variance = 0.01
+    raw = inputs.simulate_raw(sc, seed=12)
+    img = oracle.sar_rda(oracle.sar_params(sc), raw)
+    return sc, raw, img
+
+
+@pytest.mark.parametrize("fused", [False, True])
+@pytest.mark.parametrize("dtype,tol", [(C64, 1e-5), (C32H, 5e-3)])
+def test_l_band_scene_with_large_shifts(dtype, tol, fused, l_band_case):
+    sc, raw, img = l_band_case
+    got = _gpu_chain(sc, raw, dtype, fused=fused)
+    err = rel_l2(got, img)
+    assert err <= tol, err
+    for cell in sc.targets:
+        cell = tuple(cell)
+        assert quality.peak_cell(got, cell) == cell
+        assert quality.peak_cell(img, cell) == cell
+
+
+@pytest.fixture(scope="module")
 def full_scene():
     sc = inputs.x_band_scene(n_azimuth=4096, n_range=4096, n_targets=16, seed=4)
     raw = inputs.simulate_raw(sc, seed=4)
