@@ -603,13 +603,32 @@ def run_case(args):
         rd = torch.from_numpy(inputs.simulate_raw(sc, seed=4)).cuda()
         img = torch.empty_like(rd)
         p = B.sar_rda_params_create(B.sar_desc_from_scene(sc, dtype))
+        for kv in args.option:
+            B.sar_rda_set_option(p, kv.split("=")[0], int(kv.split("=")[1]))
         need = B.sar_rda_workspace_bytes(p)
         ws = torch.empty(need, dtype=torch.uint8, device="cuda")
         B.sar_rda_set_workspace(p, ws.data_ptr(), need)
         _, per = time_calls(torch, lambda: B.sar_rda_form_image(rd.data_ptr(), p, img.data_ptr(), stream.cuda_stream),
                             args.steps, args.warmup, stream)
-        B.sar_rda_params_destroy(p)
         out = summarize(per, metrics.sar_bytes(4096, 4096, dtype), peak)
+        # each step on its own, cold (a 512 MiB scratch write before every sample)
+        scratch = torch.empty(512 << 20, dtype=torch.uint8, device="cuda")
+        cold = {}
+        for label, fn in [("chain", lambda: B.sar_rda_form_image(rd.data_ptr(), p, img.data_ptr(), stream.cuda_stream))] + [
+                (f"step{s}", (lambda s=s: B.sar_rda_run_step(rd.data_ptr(), p, img.data_ptr(), s, stream.cuda_stream)))
+                for s in range(3)]:
+            ts = []
+            for i in range(9):
+                flush_l2(torch, scratch)
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(stream)
+                fn()
+                b.record(stream)
+                torch.cuda.synchronize()
+                ts.append(a.elapsed_time(b))
+            cold[label] = round(float(np.median(ts[2:])) * 1e3, 1)
+        out["cold_us"] = cold
+        B.sar_rda_params_destroy(p)
     else:
         raise SystemExit(f"unknown case {args.case}")
     out["case"] = args.case

@@ -15,25 +15,30 @@ __device__ __forceinline__ void mbar_init(uint64_t* bar, unsigned count) {
 __device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, unsigned bytes) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
 }
-// Wait for the phase with the given parity; gives up after a bounded number of polls and
-// returns false (the caller records the error and carries on: never an endless spin).
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, unsigned parity) {
+// Wait for the phase with the given parity, polling without blocking. Gives up after `limit` polls
+// (the first 64 back to back, the rest about 40 ns apart: the default limit of 2^22 is a fraction of a
+// second) and returns false; the caller records the error and winds down: never an endless spin.
+constexpr int kDefaultWaitPolls = 1 << 22;
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, unsigned parity, int limit = kDefaultWaitPolls) {
     const unsigned a = smem_u32(bar);
-    for (int i = 0; i < (1 << 22); ++i) {
+    for (int i = 0; i < limit; ++i) {
         unsigned ok;
         asm volatile(
             "{\n\t.reg .pred p;\n\t"
-            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+            "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
             "selp.u32 %0, 1, 0, p;\n\t}"
             : "=r"(ok)
             : "r"(a), "r"(parity)
             : "memory");
         if (ok) return true;
+        if (i >= 64) __nanosleep(40);
     }
     return false;
 }
 __device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+// wait until the bulk stores this thread committed have read their shared-memory source
+__device__ __forceinline__ void bulk_wait_read_all() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
 // make generic-proxy writes to shared memory visible to the asynchronous proxy
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
@@ -54,6 +59,10 @@ __device__ __forceinline__ void tma_load_2d(void* smem_dst, const void* tmap, in
             smem_u32(smem_dst)),
         "l"(tmap), "r"(x), "r"(y), "r"(smem_u32(bar))
         : "memory");
+}
+// ask L2 to fetch a box of the tensor (no shared-memory destination, no completion to wait for)
+__device__ __forceinline__ void tma_prefetch_2d(const void* tmap, int x, int y) {
+    asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global.tile [%0, {%1, %2}];" ::"l"(tmap), "r"(x), "r"(y) : "memory");
 }
 __device__ __forceinline__ void tma_store_2d(const void* tmap, int x, int y, const void* smem_src) {
     asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%1, %2}], [%3];" ::"l"(tmap), "r"(x),

@@ -50,6 +50,11 @@ using T1024 = Cfg<1024, 4, 32, 1, 1, 16, 4, 16>;
 using T2048 = Cfg<2048, 4, 32, 1, 1, 16, 8, 16>;
 using T4096 = Cfg<4096, 4, 32, 1, 1, 16, 16, 16>;
 using T8192 = Cfg<8192, 2, 32, 1, 1, 16, 32, 16>;
+// two columns per tile: half the on-chip footprint of the 4-column tiles, so that two or three CTAs share a
+// multiprocessor (used on the slab layout of the SAR chain, where a 16-byte row segment is half a granule)
+using S1024 = Cfg<1024, 2, 32, 4, 1, 16, 4, 16>;
+using S2048 = Cfg<2048, 2, 32, 2, 1, 16, 8, 16>;
+using S4096 = Cfg<4096, 2, 32, 1, 1, 16, 16, 16>;
 // wide tiles for the first pass of the two-pass split: whole 128-byte (or 64-byte) row segments
 using F64 = Cfg<64, 16, 32, 4, 1, 16, 4>;
 using F128 = Cfg<128, 16, 32, 2, 1, 16, 8>;

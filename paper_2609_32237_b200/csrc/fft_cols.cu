@@ -7,75 +7,147 @@
 
 namespace b200fft {
 
-// Column tile staged through the tensor memory accelerator on both ends: the tile arrives
-// as 2-D boxes (256 rows x W columns) in a dense [row][column] image in shared memory,
-// counted on an mbarrier; the first stage reads its registers from that image; after the
-// last stage the results are written back as the dense image and leave as TMA stores. No
-// warp-level load or store touches 16 different lines. Measured on B200 it runs exactly as
-// fast as the plain-load kernel (94 us for 4096 x 4096): the strided 32-byte access pattern
-// itself, not the way the SM issues it, sets the time (a copy-only kernel with the same
-// pattern takes 72 us). It stays selectable with the plan option "tma".
-__device__ int g_tma_timeouts = 0;   // counts mbarrier waits that ran out of polls (never expected)
+// Persistent streaming variant for the tiles that fill a multiprocessor (n = 4096 x 4 columns). With one
+// CTA per SM the plain kernel's phases run one after the other: load (10.5 K of its 25 K cycles per tile:
+// 4096 row segments of 32 bytes, sixteen cache lines per warp-level access), transform, store (another
+// 8 K). Here each CTA loops over tiles and the tensor memory accelerator moves the rows instead of the
+// load/store unit: while tile i is transformed, the boxes of tile i+1 (256 rows x W columns each) land in
+// a staging buffer beside the exchange buffer, counted on an mbarrier; the first stage reads its registers
+// from that dense image. The staging buffer holds the part of the tile that fits (12 of 16 boxes of
+// complex64, all of an fp16 tile); the remaining rows are asked into L2 at the same time and read with
+// plain loads. After the last stage the results go back to shared memory as a dense image (the exchange
+// buffer is free by then) and leave as TMA stores, which the next tile's first stage overlaps; the stores
+// must have read shared memory before the next exchange overwrites it (wait_group.read). Tensor maps cover
+// this GPU's own memory; no multicast. Every wait is bounded: a CTA whose wait runs out raises
+// g_tma_timeouts once, stops taking tiles, waits (bounded again) for the copies it still has in flight
+// and returns; the output of that call is then incomplete.
+__device__ int g_tma_timeouts = 0;   // CTAs whose wait for a copy ran out of polls (never expected)
+
+template <class C, class TIn>
+struct Stream {
+    static constexpr int BOX_ROWS = 256, NBOX = C::N / BOX_ROWS;
+    static constexpr int X_BYTES = C::N * C::W * 8;                         // exchange buffer = output image
+    static constexpr int BOX_BYTES = BOX_ROWS * C::W * TIn::ELEM_BYTES;
+    static constexpr int ROOM = 232448 - 2048 - X_BYTES;
+    static constexpr int SBOX = (ROOM / BOX_BYTES) < NBOX ? (ROOM / BOX_BYTES) : NBOX;   // boxes staged by TMA
+    static constexpr int SMEM_BYTES = X_BYTES + SBOX * BOX_BYTES;
+    static_assert(C::N % BOX_ROWS == 0 && SBOX >= 1, "whole boxes");
+    static_assert(C::CL == 1 && C::G == 1 && C::W >= 2 && C::THREADS >= NBOX, "single-CTA column tiles");
+};
 
 template <class C, bool INV, class TIn, class TOut>
-__global__ void __launch_bounds__(C::THREADS, C::MINB)
-    fft_cols_bulk_kernel(const FftArgs a, const __grid_constant__ CUtensorMap tm_in, const __grid_constant__ CUtensorMap tm_out) {
-    extern __shared__ __align__(128) float2 smem_tma[];   // TMA destinations are 128-byte aligned
+__global__ void __launch_bounds__(C::THREADS, 1)
+    fft_cols_stream_kernel(const FftArgs a, const __grid_constant__ CUtensorMap tm_in, const __grid_constant__ CUtensorMap tm_out) {
+    using L = Stream<C, TIn>;
+    extern __shared__ __align__(128) float2 smem_stream[];   // TMA destinations and sources are 128-byte aligned
     constexpr int W = C::W, N = C::N, S = C::S;
-    static_assert(C::CL == 1 && C::G == 1 && W >= 2, "single-CTA column tiles");
-    static_assert(TIn::ELEM_BYTES == 8 && TOut::ELEM_BYTES == 8, "complex64 tiles");
-    __shared__ __align__(8) uint64_t bar;
+    constexpr int XW_IN = W * TIn::ELEM_BYTES / 4, XW_OUT = W * TOut::ELEM_BYTES / 4;   // tile width in 4-byte map elements
+    __shared__ __align__(8) uint64_t bar[2];                  // [0] counts the copies; [1] is never completed
     const int t = threadIdx.x;
-    const int64_t tile = blockIdx.x;
-    float2* sm = smem_tma;
-    if (t == 0) mbar_init(&bar, 1);
+    float2* X = smem_stream;
+    char* Sb = reinterpret_cast<char*>(smem_stream) + L::X_BYTES;
+    const int polls = a.wait_polls > 0 ? a.wait_polls : kDefaultWaitPolls;
+
+    auto issue = [&](int64_t tile) {                          // thread 0: boxes of `tile` into the staging buffer
+        mbar_expect_tx(&bar[0], (unsigned)(L::SBOX * L::BOX_BYTES));
+        for (int b = 0; b < L::SBOX; ++b)
+            tma_load_2d(Sb + b * L::BOX_BYTES, &tm_in, (int)(tile * XW_IN), b * L::BOX_ROWS, &bar[0]);
+        for (int b = L::SBOX; b < L::NBOX; ++b) tma_prefetch_2d(&tm_in, (int)(tile * XW_IN), b * L::BOX_ROWS);
+    };
+    if (t == 0) {
+        mbar_init(&bar[0], 1);
+        mbar_init(&bar[1], 1);
+    }
     __syncthreads();
-    if (t == 0) mbar_expect_tx(&bar, (unsigned)(N * W * 8));
-    constexpr int BOX_ROWS = 256;
-    if (t < N / BOX_ROWS) tma_load_2d(sm + t * BOX_ROWS * W, &tm_in, (int)(tile * W * 2), t * BOX_ROWS, &bar);
-    if (!mbar_wait(&bar, 0)) atomicAdd(&g_tma_timeouts, 1);   // bounded wait: record and carry on
+    int64_t tile = blockIdx.x;
+    int in_flight = 0;                                        // thread 0: loads issued and not yet waited for
+    if (t == 0 && tile < a.tiles) {
+        issue(tile);
+        in_flight = 1;
+    }
     Engine<C> e;
     e.setup(t);
-    {
-        using G = Geo<C, 1>;
-        constexpr int V = G::V, r = G::r;
-        static_for<0, V / 2>([&](auto h_) {
-            constexpr int v = 2 * decltype(h_)::value;
-            const int c = C::template cidx<V>(t, v, 0);
-            const int q = c % W, lo = c / W;
-            static_for<0, r>([&](auto j_) {
-                constexpr int j = decltype(j_)::value;
-                const float4 u = *reinterpret_cast<const float4*>(sm + (j * G::Ls + lo) * W + q);
-                e.x[j * V + v] = make_float2(u.x, INV ? -u.y : u.y);
-                e.x[j * V + v + 1] = make_float2(u.z, INV ? -u.w : u.w);
-            });
+    unsigned phase = 0;
+    bool gave_up = false;
+    for (; tile < a.tiles; tile += gridDim.x) {
+        const int64_t next = tile + gridDim.x;
+        asm volatile("" : "+r"(e.t));                         // keep the thread index opaque per tile (register pressure)
+        using G1 = Geo<C, 1>;
+        constexpr int V = G1::V, r = G1::r;
+        static_assert(V == 2, "one register pair per first-stage slot");
+        const int c = C::template cidx<V>(e.t, 0, 0);
+        const int q = c % W, lo = c / W;
+        const int64_t gbase = tile * W;
+        auto fix = [&](int j) {
+            if constexpr (INV) {
+                e.x[j * V].y = -e.x[j * V].y;
+                e.x[j * V + 1].y = -e.x[j * V + 1].y;
+            }
+        };
+        // rows that did not fit the staging buffer: plain loads (L2 was asked for them a tile ago)
+        static_for<0, r>([&](auto j_) {
+            constexpr int j = decltype(j_)::value;
+            if constexpr ((j * G1::Ls) / L::BOX_ROWS >= L::SBOX) {
+                TIn::load2(a.in, gbase + (int64_t)(j * G1::Ls + lo) * a.dist + q, e.x[j * V], e.x[j * V + 1]);
+                fix(j);
+            }
         });
-    }
-    __syncthreads();                 // the dense image is consumed; the exchanges may overwrite it
-    e.dif(sm, a.tw);
-    __syncthreads();                 // the last exchange is consumed
-    {
-        using G = Geo<C, S>;
-        constexpr int V = G::V, r = G::r, KS = N / r;
-        static_for<0, V / 2>([&](auto h_) {
-            constexpr int v = 2 * decltype(h_)::value;
-            int b0, q;
-            e.last_index(v, b0, q);
-            static_for<0, r>([&](auto j_) {
-                constexpr int j = decltype(j_)::value;
-                const float2 p = e.x[j * V + v], w = e.x[j * V + v + 1];
-                *reinterpret_cast<float4*>(sm + (j * KS + b0) * W + q) =
-                    make_float4(p.x * a.scale, (INV ? -p.y : p.y) * a.scale, w.x * a.scale, (INV ? -w.y : w.y) * a.scale);
-            });
+        if (!mbar_wait(a.starve_wait ? &bar[1] : &bar[0], a.starve_wait ? 0u : phase, polls)) gave_up = true;
+        gave_up = __syncthreads_or(gave_up);                  // one decision per CTA
+        if (gave_up) break;
+        if (t == 0) in_flight = 0;
+        static_for<0, r>([&](auto j_) {
+            constexpr int j = decltype(j_)::value;
+            if constexpr ((j * G1::Ls) / L::BOX_ROWS < L::SBOX) {
+                TIn::load2(Sb, (j * G1::Ls + lo) * W + q, e.x[j * V], e.x[j * V + 1]);
+                fix(j);
+            }
         });
+        phase ^= 1;
+        if (t < L::NBOX) bulk_wait_read_all();                // the previous tile's stores have read the output image
+        __syncthreads();                                      // staging buffer consumed; exchange buffer free
+        if (t == 0 && next < a.tiles) {
+            issue(next);
+            in_flight = 1;
+        }
+        e.template dif<false>(X, a.tw);
+        __syncthreads();                                      // the last exchange is consumed: X becomes the output image
+        {
+            using GS = Geo<C, S>;
+            constexpr int VS = GS::V, rs = GS::r, KS = N / rs;
+            static_assert(VS == 2 && (rs == 8 || rs == 16 || rs == 32), "one register pair per last-stage slot");
+            int b0, qq;
+            e.last_index(0, b0, qq);
+            const bool scaled = a.scale != 1.0f;
+            e.template compute<S, false>(nullptr, [&](auto, auto k_, float2 pa, float2 pb) {
+                constexpr int k = decltype(k_)::value;
+                if constexpr (INV) {
+                    pa.y = -pa.y;
+                    pb.y = -pb.y;
+                }
+                if (scaled) {
+                    pa = make_float2(pa.x * a.scale, pa.y * a.scale);
+                    pb = make_float2(pb.x * a.scale, pb.y * a.scale);
+                }
+                TOut::store2(X, (k * KS + b0) * W + qq, pa, pb);
+            });
+        }
+        fence_async_smem();
+        __syncthreads();
+        if (t < L::NBOX) {
+            tma_store_2d(&tm_out, (int)(tile * XW_OUT), t * L::BOX_ROWS,
+                         reinterpret_cast<const char*>(X) + t * (L::BOX_ROWS * W * TOut::ELEM_BYTES));
+            bulk_commit();
+        }
     }
-    fence_async_smem();
-    __syncthreads();
-    if (t < N / BOX_ROWS) {
-        tma_store_2d(&tm_out, (int)(tile * W * 2), t * BOX_ROWS, sm + t * BOX_ROWS * W);
-        bulk_commit();
-        bulk_wait_all();
+    if (gave_up) {
+        if (t == 0) {
+            atomicAdd(&g_tma_timeouts, 1);
+            // copies still in flight must land before the shared memory goes away
+            if (in_flight) mbar_wait(&bar[0], phase, kDefaultWaitPolls);
+        }
     }
+    if (t < L::NBOX) bulk_wait_all();
 }
 
 // cuTensorMapEncodeTiled through the runtime's driver entry point (no link against libcuda)
@@ -93,39 +165,55 @@ static EncodeTiledFn encode_tiled_fn() {
     }
     return fn;
 }
-// rows x (ld complex64) matrix seen as fp32, boxes of box_rows rows x W complex
-static bool make_column_map(CUtensorMap* m, const void* base, int64_t rows, int64_t ld, int w, int box_rows) {
+// a rows x ld matrix of elem_bytes-sized complex elements seen as 4-byte words, boxes of box_rows rows x w elements
+static bool make_column_map(CUtensorMap* m, const void* base, int64_t rows, int64_t ld, int w, int box_rows, int elem_bytes) {
     EncodeTiledFn fn = encode_tiled_fn();
     if (!fn) return false;
-    const cuuint64_t dims[2] = {(cuuint64_t)ld * 2, (cuuint64_t)rows};
-    const cuuint64_t strides[1] = {(cuuint64_t)ld * 8};
-    const cuuint32_t box[2] = {(cuuint32_t)w * 2, (cuuint32_t)box_rows};
+    const int words = elem_bytes / 4;
+    const cuuint64_t dims[2] = {(cuuint64_t)ld * words, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)ld * elem_bytes};
+    const cuuint32_t box[2] = {(cuuint32_t)(w * words), (cuuint32_t)box_rows};
     const cuuint32_t estr[2] = {1, 1};
     return fn(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<void*>(base), dims, strides, box, estr,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <class C, bool INV>
-cudaError_t launch_cols_bulk(const FftArgs& a, cudaStream_t st) {
+template <class C, bool INV, class TI, class TO>
+cudaError_t launch_cols_stream(const FftArgs& a, cudaStream_t st) {
+    using L = Stream<C, TI>;
     static bool done[64] = {};
-    cudaError_t e = ensure_smem(fft_cols_bulk_kernel<C, INV, StoreC64, StoreC64>, C::SMEM_BYTES, done);
+    static int sms[64] = {};
+    cudaError_t e = ensure_smem(fft_cols_stream_kernel<C, INV, TI, TO>, L::SMEM_BYTES, done);
     if (e != cudaSuccess) return e;
+    // the copy engine wants 16-byte aligned bases and row pitches, and tile columns that start on 16 bytes
+    if ((reinterpret_cast<uintptr_t>(a.in) & 15) || (reinterpret_cast<uintptr_t>(a.out) & 15) ||
+        ((a.dist * TI::ELEM_BYTES) & 15) || ((a.dist * TO::ELEM_BYTES) & 15) || a.tpg != 0 || a.out_dist != 0)
+        return cudaErrorMisalignedAddress;
     CUtensorMap tin, tout;
-    if (!make_column_map(&tin, a.in, C::N, a.dist, C::W, 256) || !make_column_map(&tout, a.out, C::N, a.dist, C::W, 256))
+    if (!make_column_map(&tin, a.in, C::N, a.dist, C::W, L::BOX_ROWS, TI::ELEM_BYTES) ||
+        !make_column_map(&tout, a.out, C::N, a.dist, C::W, L::BOX_ROWS, TO::ELEM_BYTES))
         return cudaErrorNotSupported;
-    fft_cols_bulk_kernel<C, INV, StoreC64, StoreC64><<<(unsigned)a.tiles, C::THREADS, C::SMEM_BYTES, st>>>(a, tin, tout);
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    if (!sms[dev]) cudaDeviceGetAttribute(&sms[dev], cudaDevAttrMultiProcessorCount, dev);
+    const unsigned grid = (unsigned)(a.tiles < sms[dev] ? a.tiles : sms[dev]);
+    fft_cols_stream_kernel<C, INV, TI, TO><<<grid, C::THREADS, L::SMEM_BYTES, st>>>(a, tin, tout);
     g_launch_count.fetch_add(1, std::memory_order_relaxed);
     return cudaGetLastError();
 }
-template <class C, bool INV>
-constexpr KernelEntry make_bulk_entry() {
-    return KernelEntry{C::N, C::W, C::G, 77, C::THREADS, C::SMEM_BYTES, C::TW_TOTAL, INV, 0, 0,
-                       &launch_cols_bulk<C, INV>, &launch_build_tw<C>};
+template <class C, bool INV, class TS>
+constexpr KernelEntry make_stream_entry() {
+    return KernelEntry{C::N, C::W, C::G, 1, C::THREADS, Stream<C, TS>::SMEM_BYTES, C::TW_TOTAL, VAR_STREAM, INV,
+                       TS::ELEM_BYTES == 8 ? 0 : 1, TS::ELEM_BYTES == 8 ? 0 : 1,
+                       &launch_cols_stream<C, INV, TS, TS>, &launch_build_tw<C>};
 }
-static const KernelEntry k_cols_bulk[] = {make_bulk_entry<T1024, false>(), make_bulk_entry<T1024, true>(),
-                                         make_bulk_entry<T2048, false>(), make_bulk_entry<T2048, true>(),
-                                         make_bulk_entry<T4096, false>(), make_bulk_entry<T4096, true>()};
+static const KernelEntry k_cols_stream[] = {
+    make_stream_entry<T4096, false, StoreC64>(), make_stream_entry<T4096, true, StoreC64>(),
+    make_stream_entry<T4096, false, StoreC32H>(), make_stream_entry<T4096, true, StoreC32H>(),
+    make_stream_entry<T2048, false, StoreC64>(), make_stream_entry<T2048, true, StoreC64>(),
+};
 
 int tma_timeouts() {
     int v = 0;
@@ -139,37 +227,22 @@ static const KernelEntry k_cols[] = {
     B200FFT_ENTRIES_STD(T2048), B200FFT_ENTRIES_STD(T4096), B200FFT_ENTRIES_STD(T8192),
 };
 
-static int default_cluster(int n) { return 1; }
-
-const KernelEntry* find_cols_kernel(int n, bool inverse, int in_dtype, int out_dtype, int cl) {
-    if (cl == 77) {                                   // TMA-staged tiles (plan option "tma")
-        for (const KernelEntry& e : k_cols_bulk)
-            if (e.n == n && e.inverse == inverse && e.in_dtype == in_dtype && e.out_dtype == out_dtype) return &e;
+const KernelEntry* find_cols_kernel(int n, bool inverse, int in_dtype, int out_dtype, int cl, int variant) {
+    auto match = [&](const KernelEntry& e) {
+        return e.n == n && e.inverse == inverse && e.in_dtype == in_dtype && e.out_dtype == out_dtype && e.variant == variant;
+    };
+    if (variant == VAR_STREAM) {
+        for (const KernelEntry& e : k_cols_stream)
+            if (match(e)) return &e;
         return nullptr;
     }
-    const EntryList more = cols_entries_more();
-    if (cl == 1023) {                                 // wider tiles on a cluster of two CTAs
-        for (int i = 0; i < more.count; ++i) {
-            const KernelEntry& e = more.first[i];
-            if (e.cl == 2 && e.w * e.n == 32768 && e.n == n && e.inverse == inverse && e.in_dtype == in_dtype && e.out_dtype == out_dtype)
-                return &e;
-        }
-        return nullptr;
-    }
-    if (cl == 1019) {                                 // wide tiles (their entries carry w > 4)
-        for (int i = 0; i < more.count; ++i) {
-            const KernelEntry& e = more.first[i];
-            if (e.w > 4 && e.cl == 1 && e.n == n && e.inverse == inverse && e.in_dtype == in_dtype && e.out_dtype == out_dtype) return &e;
-        }
-        return nullptr;
-    }
-    if (cl == 0) cl = default_cluster(n);
+    if (cl == 0) cl = 1;
     for (const KernelEntry& e : k_cols)
-        if (e.n == n && e.cl == cl && e.inverse == inverse && e.in_dtype == in_dtype && e.out_dtype == out_dtype) return &e;
+        if (match(e) && e.cl == cl) return &e;
+    const EntryList more = cols_entries_more();
     for (int i = 0; i < more.count; ++i) {
         const KernelEntry& e = more.first[i];
-        if (e.w <= 4 && e.w * e.n != 32768 && e.n == n && e.cl == cl && e.inverse == inverse && e.in_dtype == in_dtype && e.out_dtype == out_dtype)
-            return &e;
+        if (match(e) && (variant != VAR_PLAIN || e.cl == cl)) return &e;
     }
     return nullptr;
 }

@@ -41,8 +41,29 @@ __device__ __forceinline__ void static_for(F&& f) {
 
 __host__ __device__ constexpr int ilog2(int x) { return x <= 1 ? 0 : 1 + ilog2(x >> 1); }
 
+// Complex add and subtract, optionally as one packed fp32 instruction each (sm_100 add/sub.f32x2: the
+// same two IEEE roundings as the scalar pair, so results are bit-identical, in one issue slot instead of
+// two). Measured on B200 the packed forms run at half the scalar rate per instruction, so only issue slots
+// are saved, and the aligned register pairs they need cost the large kernels more than that: N = 4096
+// +1.3 %, N = 8192 fp16 storage +2.8 %, but N = 8192 / 16384 complex64 -6 % / -7 %. Off by default;
+// -DB200FFT_PACKED_ADDS builds the packed variant.
+#ifdef B200FFT_PACKED_ADDS
+__device__ __forceinline__ float2 operator+(float2 a, float2 b) { return __fadd2_rn(a, b); }
+__device__ __forceinline__ float2 operator-(float2 a, float2 b) {
+    float2 d;
+    asm("{\n\t.reg .b64 ra, rb, rd;\n\t"
+        "mov.b64 ra, {%2, %3};\n\t"
+        "mov.b64 rb, {%4, %5};\n\t"
+        "sub.rn.f32x2 rd, ra, rb;\n\t"
+        "mov.b64 {%0, %1}, rd;\n\t}"
+        : "=f"(d.x), "=f"(d.y)
+        : "f"(a.x), "f"(a.y), "f"(b.x), "f"(b.y));
+    return d;
+}
+#else
 __device__ __forceinline__ float2 operator+(float2 a, float2 b) { return make_float2(a.x + b.x, a.y + b.y); }
 __device__ __forceinline__ float2 operator-(float2 a, float2 b) { return make_float2(a.x - b.x, a.y - b.y); }
+#endif
 __device__ __forceinline__ float2 cmul(float2 a, float2 w) {
     return make_float2(fmaf(a.x, w.x, -a.y * w.y), fmaf(a.x, w.y, a.y * w.x));
 }
@@ -777,6 +798,15 @@ struct Engine {
     template <class ST, bool CONJ>
     __device__ __forceinline__ void first_stage_dit_and_store(const float2* __restrict__ tw, void* out, int64_t base, int64_t ld,
                                                               float scale) {
+        first_stage_dit_and_store_at<ST, CONJ>(tw, out, scale, [&](int p, int q) -> int64_t {
+            return (W == 1) ? base + p : base + (int64_t)p * ld + q;
+        });
+    }
+    // The same with the caller's map from (position p, column q) of a register pair to the element index
+    // where the pair (positions p, p + 1 of a row tile; columns q, q + 1 of a column tile) is stored.
+    template <class ST, bool CONJ, class Index>
+    __device__ __forceinline__ void first_stage_dit_and_store_at(const float2* __restrict__ tw, void* out, float scale,
+                                                                 Index&& index) {
         using G = Geo<C, 1>;
         constexpr int V = G::V;
         static_assert(V >= 2, "register pairs");
@@ -784,10 +814,9 @@ struct Engine {
             constexpr int v = decltype(v_)::value, k = decltype(k_)::value;
             const int c = C::template cidx<V>(t, v, rank);
             const int q = c % W, lo = c / W;
-            const int64_t idx = (W == 1) ? base + k * G::Ls + lo : base + (int64_t)(k * G::Ls + lo) * ld + q;
             pa = make_float2(pa.x * scale, (CONJ ? -pa.y : pa.y) * scale);
             pb = make_float2(pb.x * scale, (CONJ ? -pb.y : pb.y) * scale);
-            ST::store2(out, idx, pa, pb);
+            ST::store2(out, index(k * G::Ls + lo, q), pa, pb);
         });
     }
 
@@ -888,7 +917,27 @@ struct FftArgs {
     int64_t dist;    // rows: elements between transforms; columns: elements between rows (ld)
     float scale;
     int prefetch_ahead;   // rows: tiles ahead whose input one thread asks L2 to fetch (0 = off)
+    // Column tiles of a slab image (see slab_index): tpg = tiles per slab, slab_stride = elements per
+    // slab, dist = columns per slab. tpg == 0: a plain row-major matrix (tile t starts at column t * W).
+    int64_t tpg = 0, slab_stride = 0;
+    // Output geometry where it differs from the input's (out_dist == 0: the same as the input's).
+    int64_t out_dist = 0, out_tpg = 0, out_slab_stride = 0;
+    // Kernels that wait on asynchronous copies: polls before a wait gives up (0 = the default), and a test
+    // knob that makes the consumer wait on a barrier nothing ever completes, so that the give-up path runs.
+    int wait_polls = 0, starve_wait = 0;
 };
+
+// Slab layout of an image with `rows` rows and G columns per granule: columns are grouped G at a time
+// and every group (slab) is stored as its own contiguous rows x G matrix, so that the element of row k
+// and column n lives at ((n / G) * rows + k) * G + n % G. A tile of W <= G adjacent columns is then
+// row segments at a pitch of G elements inside one contiguous slab.
+__host__ __device__ __forceinline__ int64_t slab_index(int64_t k, int64_t n, int64_t rows, int g) {
+    return ((n / g) * rows + k) * g + (n % g);
+}
+// first element of column tile `tile` (W columns wide)
+__device__ __forceinline__ int64_t column_tile_base(int64_t tile, int w, int64_t tpg, int64_t slab_stride) {
+    return tpg ? (tile / tpg) * slab_stride + (tile % tpg) * w : tile * w;
+}
 
 // Ask L2 to start fetching `bytes` contiguous bytes (a multiple of 16, 16-byte aligned).
 __device__ __forceinline__ void prefetch_l2_bulk(const void* p, unsigned bytes) {
@@ -905,7 +954,14 @@ __global__ void __launch_bounds__(C::THREADS, C::MINB) fft_kernel(const FftArgs 
     const bool active = tile < a.tiles;
     if (!active) tile = a.tiles - 1;          // keep the barriers uniform; results discarded
     float2* sm = smem_dyn + g * C::LOCAL_ELEMS;
-    const int64_t base = (C::W == 1) ? tile * a.dist : tile * C::W;
+    const int64_t base = (C::W == 1) ? tile * a.dist : column_tile_base(tile, C::W, a.tpg, a.slab_stride);
+    int64_t obase = base, odist = a.dist;
+    if constexpr (C::W > 1) {
+        if (a.out_dist) {
+            obase = column_tile_base(tile, C::W, a.out_tpg, a.out_slab_stride);
+            odist = a.out_dist;
+        }
+    }
     Engine<C> e;
     e.setup(t);
     if constexpr (C::W == 1 && C::G == 1) {
@@ -921,7 +977,7 @@ __global__ void __launch_bounds__(C::THREADS, C::MINB) fft_kernel(const FftArgs 
     }
     e.template load_first<TIn, INV>(a.in, base, a.dist);
     e.template dif<false>(sm, a.tw);
-    if (active) e.template last_stage_and_store<TOut, INV>(a.out, base, a.dist, a.scale);
+    if (active) e.template last_stage_and_store<TOut, INV>(a.out, obase, odist, a.scale);
 }
 
 // Builds the per-stage twiddle rows of a configuration in float64, rounds once to fp32:

@@ -154,7 +154,7 @@ cudaError_t launch_staged(const FftArgs& a, cudaStream_t st) {
 }
 template <class C, bool INV, class TI, class TO, int CPS>
 constexpr KernelEntry make_staged_entry() {
-    return KernelEntry{C::N, C::W, C::G, 1017, C::THREADS, Staged<C, TI, CPS>::SMEM_BYTES, C::TW_TOTAL, INV,
+    return KernelEntry{C::N, C::W, C::G, 1, C::THREADS, Staged<C, TI, CPS>::SMEM_BYTES, C::TW_TOTAL, VAR_STAGED, INV,
                        TI::ELEM_BYTES == 8 ? 0 : 1, TO::ELEM_BYTES == 8 ? 0 : 1,
                        &launch_staged<C, INV, TI, TO, CPS>, &launch_build_tw<C>};
 }
@@ -183,27 +183,21 @@ static int default_cluster(int n, int64_t batch) {
     return 1;
 }
 
-const KernelEntry* find_rows_kernel(int n, bool inverse, int in_dtype, int out_dtype, int cl, int64_t batch) {
-    if (cl == 1015 || cl == 1016) {                   // test knobs: 1015 = all first-stage twiddle rows from
-                                                      // the table (n = 4096); 1016 = four-stage n = 16384
-        const EntryList l = rows_entries_large();
-        for (int i = 0; i < l.count; ++i) {
-            const KernelEntry& e = l.first[i];
-            if (e.cl == cl && e.n == n && e.inverse == inverse && e.in_dtype == in_dtype && e.out_dtype == out_dtype) return &e;
-        }
-        return nullptr;
-    }
-    if (cl == 1017) {                                 // staged persistent variant (plan option "staged")
+const KernelEntry* find_rows_kernel(int n, bool inverse, int in_dtype, int out_dtype, int cl, int64_t batch, int variant) {
+    auto match = [&](const KernelEntry& e) {
+        return e.n == n && e.inverse == inverse && e.in_dtype == in_dtype && e.out_dtype == out_dtype && e.variant == variant;
+    };
+    if (variant == VAR_STAGED) {
         for (const KernelEntry& e : k_rows_staged)
-            if (e.n == n && e.inverse == inverse && e.in_dtype == in_dtype && e.out_dtype == out_dtype) return &e;
+            if (match(e)) return &e;
         return nullptr;
     }
-    if (cl == 0) cl = default_cluster(n, batch);
+    if (variant == VAR_PLAIN && cl == 0) cl = default_cluster(n, batch);
     const EntryList lists[3] = {rows_entries_small(), rows_entries_large(), rows_entries_cluster()};
     for (const EntryList& l : lists)
         for (int i = 0; i < l.count; ++i) {
             const KernelEntry& e = l.first[i];
-            if (e.n == n && e.cl == cl && e.inverse == inverse && e.in_dtype == in_dtype && e.out_dtype == out_dtype) return &e;
+            if (match(e) && (variant != VAR_PLAIN || e.cl == cl)) return &e;
         }
     return nullptr;
 }

@@ -1,5 +1,5 @@
 // Single-pass row kernels, N = 4096 .. 16384 (one transform per CTA), and the alternative
-// factorisations kept as test knobs (entries with cl = 1015, 1016).
+// factorisations kept as test knobs (variants VAR_TW_TABLE, VAR_FOUR_STAGE).
 #include "configs.h"
 #include "registry.h"
 
@@ -8,7 +8,7 @@ namespace b200fft {
 template <class C, bool INV, class TI, class TO>
 constexpr KernelEntry make_alt_entry(int knob) {
     KernelEntry e = make_entry<C, INV, TI, TO>();
-    e.cl = knob;
+    e.variant = knob;
     return e;
 }
 #define B200FFT_ENTRIES_ALT(C, K)                                                                      \
@@ -17,7 +17,7 @@ constexpr KernelEntry make_alt_entry(int knob) {
 
 static const KernelEntry k_rows_large[] = {
     B200FFT_ENTRIES_STD(R4096), B200FFT_ENTRIES_STD(R8192), B200FFT_ENTRIES_STD(R16384),
-    B200FFT_ENTRIES_ALT(R4096t15, 1015), B200FFT_ENTRIES_ALT(R16384s4, 1016),
+    B200FFT_ENTRIES_ALT(R4096t15, VAR_TW_TABLE), B200FFT_ENTRIES_ALT(R16384s4, VAR_FOUR_STAGE),
 };
 
 EntryList rows_entries_large() { return EntryList{k_rows_large, (int)(sizeof(k_rows_large) / sizeof(k_rows_large[0]))}; }

@@ -20,6 +20,8 @@ struct b200fft_plan_s {
     Layout layout;
     bool four_step;
     int cluster;                 // CTAs per tile requested by the "cluster" option (0 = default)
+    int variant;                 // kernel family forced by an option (VAR_PLAIN = the default rules)
+    int wait_polls, starve_wait; // test knobs of the kernels that wait on asynchronous copies
     int prefetch_ahead;          // "prefetch" option: tiles ahead to prefetch into L2 (-1 = default)
     bool via_transpose;          // "via_transpose" option (columns): transpose, row transforms, transpose back
     const KernelEntry* rows_kernel;   // its row variant and table
@@ -27,6 +29,7 @@ struct b200fft_plan_s {
     const BfpEntry* bfp;         // block-floating-point variant and its table, built on first use
     float2* tw_bfp;
     int staged;                  // "staged" option: persistent kernel fed by the copy engine (-1 = default)
+    int stream;                  // "stream" option (columns): 0 forbids the streaming kernel, -1 = default rules
     const KernelEntry* kernel;   // single-pass variant
     float2* tw;                  // its twiddle rows (device)
     int device;
@@ -49,27 +52,36 @@ static int elem_bytes(int dtype) { return dtype == B200FFT_C64 ? 8 : 4; }
 
 static int build_single_pass(b200fft_plan_s* p) {
     const bool inv = p->direction == B200FFT_INVERSE;
-    int cl = p->cluster;
-    if (p->layout == LAYOUT_ROWS && cl == 0) {
+    const int cl = p->cluster;
+    int variant = p->variant;
+    const KernelEntry* k = nullptr;
+    if (p->layout == LAYOUT_ROWS && variant == VAR_PLAIN && cl == 0) {
         // Persistent staged kernel: measured on B200 at n = 16384 with fp16 storage, 379 -> 342 us for
         // 8192 transforms; with fp32 storage it is slower than the plain kernel (455 against 447 us:
         // only half of the tile can wait beside the exchange buffer), so there it is only taken on request.
         const bool by_default = p->n == 16384 && p->dtype == B200FFT_C32H && p->batch >= 2 * (int64_t)p->sms;
-        if (p->staged == 1 || (p->staged == -1 && by_default)) cl = 1017;
+        if (p->staged == 1 || (p->staged == -1 && by_default)) variant = VAR_STAGED;
     }
-    const KernelEntry* k = nullptr;
-    if (p->layout == LAYOUT_COLS && cl == 0) {          // wide tiles where they exist and divide the batch:
-        k = find_cols_kernel((int)p->n, inv, p->dtype, p->dtype, 1019);       // 16 columns for n <= 1024
+    if (p->layout == LAYOUT_COLS && variant == VAR_PLAIN && cl == 0) {
+        // default rules, widest first: 16-column tiles for n <= 1024 where they divide the batch ...
+        k = find_cols_kernel((int)p->n, inv, p->dtype, p->dtype, 0, VAR_WIDE);
         if (k && p->batch % k->w) k = nullptr;
-        if (!k && !(p->n == 2048 && p->dtype == B200FFT_C64)) {                // a cluster of two CTAs for n >= 2048
-            // (measured: n = 2048 complex64 80 us with 4-column tiles against 84 us, fp16 storage 80 -> 70 us)
-            k = find_cols_kernel((int)p->n, inv, p->dtype, p->dtype, 1023);
+        // ... the persistent streaming kernel for tiles that fill a multiprocessor, when there is more than one
+        // tile per multiprocessor to overlap ...
+        if (!k && p->stream != 0 && p->batch / 4 > p->sms) {
+            k = find_cols_kernel((int)p->n, inv, p->dtype, p->dtype, 0, VAR_STREAM);
+            if (k && (p->batch % k->w || k->n < 4096)) k = nullptr;
+        }
+        // ... else a tile twice as wide on a cluster of two CTAs for n >= 2048
+        // (measured: n = 2048 complex64 80 us with 4-column tiles against 84 us, fp16 storage 80 -> 70 us)
+        if (!k && !(p->n == 2048 && p->dtype == B200FFT_C64)) {
+            k = find_cols_kernel((int)p->n, inv, p->dtype, p->dtype, 0, VAR_WIDE_CLUSTER);
             if (k && p->batch % k->w) k = nullptr;
         }
     }
     if (!k)
-        k = (p->layout == LAYOUT_ROWS) ? find_rows_kernel((int)p->n, inv, p->dtype, p->dtype, cl, p->batch)
-                                       : find_cols_kernel((int)p->n, inv, p->dtype, p->dtype, cl);
+        k = (p->layout == LAYOUT_ROWS) ? find_rows_kernel((int)p->n, inv, p->dtype, p->dtype, cl, p->batch, variant)
+                                       : find_cols_kernel((int)p->n, inv, p->dtype, p->dtype, cl, variant);
     if (!k) return B200FFT_ERR_UNSUPPORTED;
     if (p->layout == LAYOUT_COLS && p->batch % k->w) return B200FFT_ERR_UNSUPPORTED;
     p->kernel = k;                  // the table depends on the factorisation: always rebuilt
@@ -82,6 +94,18 @@ static int build_single_pass(b200fft_plan_s* p) {
     if (p->kernel->build_tw(p->tw, 0) != cudaSuccess) return B200FFT_ERR_CUDA;
     if (cudaStreamSynchronize(0) != cudaSuccess) return B200FFT_ERR_CUDA;
     return B200FFT_OK;
+}
+
+// set one selection field, rebuild, and put the old value back if no such kernel exists
+static int reselect(b200fft_plan_s* p, int* field, int value) {
+    const int old = *field;
+    *field = value;
+    int rc = build_single_pass(p);
+    if (rc != B200FFT_OK) {
+        *field = old;
+        build_single_pass(p);
+    }
+    return rc;
 }
 
 static void release(b200fft_plan_s* p) {
@@ -143,6 +167,8 @@ extern "C" int fft_plan_create(fft_plan_t* plan, int64_t n, int64_t batch, int64
     p->direction = direction; p->dtype = storage_dtype; p->layout = layout;
     p->prefetch_ahead = -1;
     p->staged = -1;
+    p->stream = -1;
+    p->variant = VAR_PLAIN;
     if (cudaGetDevice(&p->device) != cudaSuccess) { delete p; return B200FFT_ERR_CUDA; }
     p->sms = 148;
     cudaDeviceGetAttribute(&p->sms, cudaDevAttrMultiProcessorCount, p->device);
@@ -199,7 +225,7 @@ extern "C" int fft_plan_set_option(fft_plan_t p, const char* key, int64_t value)
         }
         if (!p->rows_kernel) {
             const KernelEntry* k = find_rows_kernel((int)p->n, p->direction == B200FFT_INVERSE, p->dtype, p->dtype, 0, p->batch);
-            if (!k || k->cl == 1017) k = find_rows_kernel((int)p->n, p->direction == B200FFT_INVERSE, p->dtype, p->dtype, 1, p->batch);
+            if (!k) k = find_rows_kernel((int)p->n, p->direction == B200FFT_INVERSE, p->dtype, p->dtype, 1, p->batch);
             if (!k) return B200FFT_ERR_UNSUPPORTED;
             if (cudaMalloc(&p->tw_rows, sizeof(float2) * (size_t)k->tw_total) != cudaSuccess) {
                 cudaGetLastError();
@@ -214,36 +240,39 @@ extern "C" int fft_plan_set_option(fft_plan_t p, const char* key, int64_t value)
     }
     if (std::strcmp(key, "staged") == 0) {
         if (p->four_step || p->layout != LAYOUT_ROWS || value < -1 || value > 1) return B200FFT_ERR_UNSUPPORTED;
-        const int old = p->staged;
-        p->staged = (int)value;
-        int rc = build_single_pass(p);
-        if (rc != B200FFT_OK) {
-            p->staged = old;
-            build_single_pass(p);
-            return rc;
-        }
-        return B200FFT_OK;
+        return reselect(p, &p->staged, (int)value);
     }
-    if (std::strcmp(key, "tma") == 0) {
-        if (p->four_step || p->layout != LAYOUT_COLS || p->dtype != B200FFT_C64) return B200FFT_ERR_UNSUPPORTED;
-        const int old = p->cluster;
-        p->cluster = value ? 77 : 0;
-        int rc = build_single_pass(p);
-        if (rc != B200FFT_OK) {
-            p->cluster = old;
+    if (std::strcmp(key, "stream") == 0 || std::strcmp(key, "tma") == 0) {
+        // 1: the persistent streaming column kernel; 0: never; -1: the default rules
+        if (p->four_step || p->layout != LAYOUT_COLS || value < -1 || value > 1) return B200FFT_ERR_UNSUPPORTED;
+        if (value == 1) {
+            int rc = reselect(p, &p->variant, VAR_STREAM);
+            if (rc == B200FFT_OK) p->cluster = 0;
             return rc;
         }
-        return B200FFT_OK;
+        p->variant = VAR_PLAIN;
+        return reselect(p, &p->stream, (int)value);
     }
     if (std::strcmp(key, "cluster") == 0) {
         if (p->four_step || p->n > 32768) return B200FFT_ERR_UNSUPPORTED;
-        const int old = p->cluster;
-        p->cluster = (int)value;
-        int rc = build_single_pass(p);
-        if (rc != B200FFT_OK) {
-            p->cluster = old;
-            return rc;
-        }
+        if (value != 0 && value != 1 && value != 2 && value != 4) return B200FFT_ERR_INVALID_ARG;
+        p->variant = VAR_PLAIN;
+        return reselect(p, &p->cluster, (int)value);
+    }
+    if (std::strcmp(key, "alt_factorisation") == 0) {
+        // test knob: the other compiled factorisation of a rows plan (n = 4096 with every first-stage
+        // twiddle row loaded from its table; n = 16384 as 16 x 4 x 16 x 16)
+        if (p->four_step || p->layout != LAYOUT_ROWS) return B200FFT_ERR_UNSUPPORTED;
+        if (!value) return reselect(p, &p->variant, VAR_PLAIN);
+        return reselect(p, &p->variant, p->n == 4096 ? VAR_TW_TABLE : VAR_FOUR_STAGE);
+    }
+    if (std::strcmp(key, "wait_polls") == 0) {
+        if (value < 0 || value > (1 << 30)) return B200FFT_ERR_INVALID_ARG;
+        p->wait_polls = (int)value;
+        return B200FFT_OK;
+    }
+    if (std::strcmp(key, "starve_wait") == 0) {
+        p->starve_wait = value != 0;
         return B200FFT_OK;
     }
     return B200FFT_ERR_INVALID_ARG;
@@ -338,7 +367,9 @@ static int launch_single_pass(b200fft_plan_s* p, const void* in, void* out, int6
     a.out = out;
     a.tw = p->tw;
     a.prefetch_ahead = 0;
-    if (p->layout == LAYOUT_ROWS && p->kernel->cl >= 1 && p->kernel->cl <= 8 && p->kernel->g == 1) {
+    a.wait_polls = p->wait_polls;
+    a.starve_wait = p->starve_wait;
+    if (p->layout == LAYOUT_ROWS && p->kernel->variant != VAR_STAGED && p->kernel->g == 1) {
         // default: for tiles that fill an SM (one CTA resident), the tile one full wave ahead;
         // measured on B200: +13 % at n = 16384 rows, nothing to gain at n = 8192 and below,
         // and a loss for column tiles (their time goes to the lock-step compute, not the load)

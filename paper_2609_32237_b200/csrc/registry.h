@@ -9,8 +9,21 @@ namespace b200fft {
 
 extern std::atomic<int64_t> g_launch_count;
 
+// Which kernel family an entry belongs to. The default family is the plain kernel for its size and
+// cluster width; the others are alternatives that a plan option or a default rule selects.
+enum Variant : int {
+    VAR_PLAIN = 0,
+    VAR_TW_TABLE,        // rows, n = 4096: every first-stage twiddle row loaded from the table (test knob)
+    VAR_FOUR_STAGE,      // rows, n = 16384 as 16 x 4 x 16 x 16 (test knob)
+    VAR_STAGED,          // rows: persistent kernel, next transform staged by untiled bulk copies
+    VAR_STREAM,          // columns: persistent kernel, tiles staged in and out by the tensor memory accelerator
+    VAR_WIDE,            // columns: tiles wider than four columns on one CTA
+    VAR_WIDE_CLUSTER,    // columns: tiles of 32768 / n columns shared by a cluster of two CTAs
+};
+
 struct KernelEntry {
     int n, w, g, cl, threads, smem_bytes, tw_total;
+    int variant;
     bool inverse;
     int in_dtype, out_dtype;                 // 0 = c64, 1 = c32h
     cudaError_t (*launch)(const FftArgs&, cudaStream_t);
@@ -71,7 +84,7 @@ cudaError_t launch_build_tw(float2* tw, cudaStream_t st) {
 
 template <class C, bool INV, class TI, class TO>
 constexpr KernelEntry make_entry() {
-    return KernelEntry{C::N, C::W, C::G, C::CL, C::THREADS, C::SMEM_BYTES, C::TW_TOTAL, INV,
+    return KernelEntry{C::N, C::W, C::G, C::CL, C::THREADS, C::SMEM_BYTES, C::TW_TOTAL, VAR_PLAIN, INV,
                        TI::ELEM_BYTES == 8 ? 0 : 1, TO::ELEM_BYTES == 8 ? 0 : 1,
                        &launch_fft<C, INV, TI, TO>, &launch_build_tw<C>};
 }
@@ -103,14 +116,16 @@ EntryList rows_entries_large();     // N = 4096 .. 16384 and the alternative fac
 EntryList rows_entries_cluster();   // transforms shared by a cluster of CTAs
 EntryList cols_entries_more();      // column tiles on clusters, wide column tiles
 
-// cl: CTAs per tile (cluster size); 0 picks the default variant for that size
+// cl: CTAs per tile (cluster size); 0 picks the default for that size and batch (plain kernels only)
 const KernelEntry* find_rows_kernel(int n, bool inverse, int in_dtype, int out_dtype, int cl = 0,
-                                    int64_t batch = (int64_t)1 << 40);
-const KernelEntry* find_cols_kernel(int n, bool inverse, int in_dtype, int out_dtype, int cl = 0);
+                                    int64_t batch = (int64_t)1 << 40, int variant = VAR_PLAIN);
+const KernelEntry* find_cols_kernel(int n, bool inverse, int in_dtype, int out_dtype, int cl = 0, int variant = VAR_PLAIN);
+// column tiles of the SAR chain on the slab layout: w = 2 or 4 columns, any pair of storage types
+const KernelEntry* find_sar_cols_kernel(int n, int w, bool inverse, int in_dtype, int out_dtype);
 // out[c * ld_out + r] = in[r * ld_in + c]; elem_bytes 8 (complex64) or 4 (complex half)
 cudaError_t transpose_launch(const void* in, void* out, int rows, int cols, int64_t ld_in, int64_t ld_out, int elem_bytes,
                              cudaStream_t st);
-int tma_timeouts();   // mbarrier waits of the TMA column variant that ran out of polls since load
+int tma_timeouts();   // CTAs of the streaming column kernel whose wait for a copy ran out of polls since load
 int rows_stage_timeouts();   // the same for the staged persistent row kernels
 
 }  // namespace b200fft

@@ -8,6 +8,13 @@
 //           output scaled by 1/n_azimuth (the paper's fixed-shift schedule)
 //   step 2  fused range cell migration correction (8-tap sinc), azimuth filter
 //           exp(+j 4 pi R0 (D - 1) / lambda) and inverse azimuth FFT on column tiles
+// Between the steps the image lives in the caller's workspace. Its layout is the library's own
+// choice, and by default it is the slab layout of fft_core.cuh with 32-byte granules (4 complex64
+// or 8 complex-half range bins): every column tile of the azimuth transforms is then row segments
+// inside one contiguous slab instead of 32-byte pieces at a pitch of a whole image row, range
+// compression still writes whole sectors, and step 2 runs as a row-wise pass over slabs (RCMC +
+// filter, slab to slab) followed by the inverse column transform that writes the row-major image.
+// The row-major intermediate of the first design stays selectable (option "layout" = 0).
 // The filter and the migration are affine in the range index with per-Doppler-bin
 // coefficients, built once in float64. The paper's four numerical fixes are kept:
 // baseband filter (D - 1); phase in cycles with a split that makes the fp32
@@ -40,10 +47,12 @@ struct SarArgs {
     int64_t ld;          // row pitch in elements (n_range)
     int nr;
     float scale;
+    int na;              // rows of the image (n_azimuth)
 };
 
 // ---------------------------------------------------------------- step 0
-template <class C, class TOut>
+// SLAB: the output goes to the slab layout (granules of 32 bytes) instead of row-major.
+template <class C, class TOut, bool SLAB>
 __global__ void __launch_bounds__(C::THREADS, C::MINB) sar_range_compress_kernel(const SarArgs a) {
     extern __shared__ __align__(16) float2 smem_dyn[];
     static_assert(C::W == 1, "range compression works on contiguous rows");
@@ -78,7 +87,16 @@ __global__ void __launch_bounds__(C::THREADS, C::MINB) sar_range_compress_kernel
         });
     }
     e.template dit<false>(sm, a.tw);
-    if (active) e.template first_stage_dit_and_store<TOut, true>(a.tw, a.out, base, a.ld, 1.0f);
+    if (!active) return;
+    if constexpr (SLAB) {
+        constexpr int GS = 32 / TOut::ELEM_BYTES;
+        const int64_t na = a.na;
+        e.template first_stage_dit_and_store_at<TOut, true>(a.tw, a.out, 1.0f, [&](int p, int) -> int64_t {
+            return ((int64_t)(p / GS) * na + tile) * GS + (p % GS);
+        });
+    } else {
+        e.template first_stage_dit_and_store<TOut, true>(a.tw, a.out, base, a.ld, 1.0f);
+    }
 }
 
 // ---------------------------------------------------------------- step 2
@@ -159,7 +177,7 @@ __host__ __device__ constexpr int rcmc_smem_bytes() {
     return (st > C::SMEM_BYTES ? st : C::SMEM_BYTES) + C::N * 4;   // + one window start per row
 }
 
-template <class C, class TIn>
+template <class C, class TIn, bool SLAB>
 __global__ void __launch_bounds__(C::THREADS, 1) sar_rcmc_filter_ifft_kernel(const SarArgs a) {
     extern __shared__ __align__(16) float2 smem_dyn[];
     constexpr int W = C::W;
@@ -204,7 +222,9 @@ __global__ void __launch_bounds__(C::THREADS, 1) sar_rcmc_filter_ifft_kernel(con
             const int k = j * ROWS + row;
             const int col = wstart[k] + gr * GRAN;
             const bool valid = col >= 0 && col + GRAN <= a.nr;
-            cp_async_16(stg + stg_index(j & 3, row, gr * GRAN), in + (int64_t)k * a.ld + (valid ? col : 0), valid);
+            const int cc = valid ? col : 0;                  // a 16-byte piece never straddles a 32-byte granule
+            const int64_t src = SLAB ? slab_index(k, cc, a.na, 32 / EB) : (int64_t)k * a.ld + cc;
+            cp_async_16(stg + stg_index(j & 3, row, gr * GRAN), in + src, valid);
         }
     };
 
@@ -378,6 +398,130 @@ __global__ void __launch_bounds__(RcmcRows::TPB) sar_rcmc_filter_rows_kernel(con
     }
 }
 
+// ---------------------------------------------------------------- step 2a on the slab layout
+// Range cell migration correction and azimuth filter, slab image to slab image. A CTA works on 32
+// consecutive Doppler bins (the lanes of every warp) by NC consecutive range bins (four per thread);
+// in the slab layout the 32 rows of one granule column are one contiguous kilobyte, so the window
+// is staged with whole-line loads, the results leave as whole lines, and a lane's taps sit in its
+// own shared-memory column (conflict-free whatever the row's shift is). The window of every CTA
+// starts at its smallest integer shift; how far the shift may spread inside a CTA is checked when
+// the parameters are created.
+template <class TIn, class TOut>
+struct RcmcSlab {
+    static constexpr int ROWS = 32, NC = 64, HALO = 32, NS = NC + HALO;
+    static constexpr int THREADS = NC / 4 * 32;
+    static constexpr int GI = 32 / TIn::ELEM_BYTES, GO = 32 / TOut::ELEM_BYTES;
+    static constexpr int MAX_SPREAD = HALO - 8 - 6;     // allowed (largest - smallest) integer shift in a CTA
+};
+
+template <class TIn, class TOut>
+__global__ void __launch_bounds__(RcmcSlab<TIn, TOut>::THREADS) sar_rcmc_filter_slab_kernel(const SarArgs a) {
+    using L = RcmcSlab<TIn, TOut>;
+    constexpr int NS = L::NS, GI = L::GI, GO = L::GO;
+    __shared__ __align__(16) float2 win[NS * 32];       // [sample][row]
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    const int kblocks = a.na / 32;
+    const int k0 = (blockIdx.x % kblocks) * 32, n0 = (blockIdx.x / kblocks) * L::NC;
+    const int k = k0 + lane;
+    const float4 mg = __ldg(a.tab.mig + k);
+    int s0;
+    {   // |f| is monotonic over the 32 rows (a block never straddles n_azimuth / 2) and the shift grows
+        // with the range bin: the smallest shift is at the first range bin of the first or last row
+        int ia, ib;
+        float mu;
+        migration(__ldg(a.tab.mig + k0), n0, ia, mu);
+        migration(__ldg(a.tab.mig + k0 + 31), n0, ib, mu);
+        s0 = (n0 + min(ia, ib) - 3) & ~(GI - 1);        // floors for negative values too
+    }
+    {   // stage the window: 16-byte pieces, a warp takes one half of the granules of 32 rows
+        const char* in = reinterpret_cast<const char*>(a.in);
+        const int slab0 = s0 / GI;                       // exact: s0 is a multiple of GI
+        const int nslabs = a.nr / GI;
+        constexpr int PIECES = (NS / GI) * 64;
+        for (int id = threadIdx.x; id < PIECES; id += L::THREADS) {
+            const int rel = id >> 6, half = (id >> 5) & 1, row = id & 31;
+            const int slab = slab0 + rel;
+            uint4 v = make_uint4(0u, 0u, 0u, 0u);       // samples outside the row read as zero
+            if (slab >= 0 && slab < nslabs)
+                v = __ldg(reinterpret_cast<const uint4*>(in + ((int64_t)slab * a.na + k0 + row) * 32 + half * 16));
+            float2* dst = win + (rel * GI + half * (GI / 2)) * 32 + row;
+            if constexpr (TIn::ELEM_BYTES == 8) {
+                dst[0] = make_float2(__uint_as_float(v.x), __uint_as_float(v.y));
+                dst[32] = make_float2(__uint_as_float(v.z), __uint_as_float(v.w));
+            } else {
+                dst[0] = __half22float2(*reinterpret_cast<const __half2*>(&v.x));
+                dst[32] = __half22float2(*reinterpret_cast<const __half2*>(&v.y));
+                dst[64] = __half22float2(*reinterpret_cast<const __half2*>(&v.z));
+                dst[96] = __half22float2(*reinterpret_cast<const __half2*>(&v.w));
+            }
+        }
+    }
+    __syncthreads();
+    const int n = n0 + 4 * w;
+    int i0[4];
+    float mu[4];
+    migration(mg, n, i0[0], mu[0]);
+    const float g = mg.x + mg.y;
+#pragma unroll
+    for (int p = 1; p < 4; ++p) {                        // one range bin on: the migration grows by the slope
+        mu[p] = mu[p - 1] + g;
+        i0[p] = i0[p - 1];
+        if (mu[p] >= 1.0f) {
+            mu[p] -= 1.0f;
+            i0[p] += 1;
+        }
+    }
+    const float2* col = win + lane;
+    float2 acc[4];
+    auto taps = [&](int p, const float2* u) {            // u[0..7]: the eight samples of pixel p, tap j = -3 first
+        float wt[8];
+        sinc8_weights_rcp(mu[p], wt);
+        float2 s = make_float2(0.f, 0.f);
+#pragma unroll
+        for (int tap = 0; tap < 8; ++tap) {
+            const float ww = ((tap - 3) & 1) ? -wt[tap] : wt[tap];
+            s.x = fmaf(ww, u[tap].x, s.x);
+            s.y = fmaf(ww, u[tap].y, s.y);
+        }
+        acc[p] = s;
+    };
+    if (i0[3] == i0[0]) {                                // the usual case: one window of 11 samples serves all four
+        const int o = min(max(n + i0[0] - 3 - s0, 0), NS - 11);
+        float2 u[11];
+#pragma unroll
+        for (int i = 0; i < 11; ++i) u[i] = col[(o + i) * 32];
+#pragma unroll
+        for (int p = 0; p < 4; ++p) taps(p, u + p);
+    } else {
+#pragma unroll
+        for (int p = 0; p < 4; ++p) {
+            const int o = min(max(n + p + i0[p] - 3 - s0, 0), NS - 8);
+            float2 u[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) u[i] = col[(o + i) * 32];
+            taps(p, u);
+        }
+    }
+    float2 f = filter_phase(__ldg(a.tab.phs + k), n);
+    const float2 step = __ldg(a.tab.stp + k);
+#pragma unroll
+    for (int p = 0; p < 4; ++p) {
+        acc[p] = cmul(acc[p], f);
+        if (p < 3) f = cmul(f, step);                    // one more range bin: times exp(j 2 pi B)
+    }
+    if constexpr (TOut::ELEM_BYTES == 8) {
+        float4* o = reinterpret_cast<float4*>(reinterpret_cast<float2*>(a.out) + slab_index(k, n, a.na, GO));
+        o[0] = make_float4(acc[0].x, acc[0].y, acc[1].x, acc[1].y);
+        o[1] = make_float4(acc[2].x, acc[2].y, acc[3].x, acc[3].y);
+    } else {
+        __half2 h[4];
+#pragma unroll
+        for (int p = 0; p < 4; ++p) h[p] = __float22half2_rn(acc[p]);
+        *reinterpret_cast<uint4*>(reinterpret_cast<__half2*>(a.out) + slab_index(k, n, a.na, GO)) =
+            *reinterpret_cast<const uint4*>(h);
+    }
+}
+
 // ---------------------------------------------------------------- tables (float64, built once)
 // H[k] = conj( sum_i h[i] exp(-2 pi i k i / nr) ) / nr,  h[i] = exp(j pi K (i/fs)^2), i = -P/2 .. P-P/2-1
 __global__ void sar_build_matched_filter(float2* H, int nr, int pulse_samples, double kappa) {
@@ -433,44 +577,78 @@ __global__ void sar_build_doppler_tables(float4* mig, float4* phs, float2* stp, 
 }
 
 // ---------------------------------------------------------------- host side
-template <class C, class TOut>
+template <class C, class TOut, bool SLAB>
 cudaError_t launch_range(const SarArgs& a, cudaStream_t st) {
     static bool done[64] = {};
-    cudaError_t e = ensure_smem(sar_range_compress_kernel<C, TOut>, C::SMEM_BYTES, done);
+    cudaError_t e = ensure_smem(sar_range_compress_kernel<C, TOut, SLAB>, C::SMEM_BYTES, done);
     if (e != cudaSuccess) return e;
-    return launch_tiles<C>(sar_range_compress_kernel<C, TOut>, a, a.tiles, st);
+    return launch_tiles<C>(sar_range_compress_kernel<C, TOut, SLAB>, a, a.tiles, st);
 }
-template <class C, class TIn>
+template <class C, class TIn, bool SLAB>
 cudaError_t launch_rcmc(const SarArgs& a, cudaStream_t st) {
     static bool done[64] = {};
     constexpr int smem = rcmc_smem_bytes<C, TIn>();
     static_assert(smem <= 227 * 1024, "tile + staging must fit one CTA's shared memory");
-    cudaError_t e = ensure_smem(sar_rcmc_filter_ifft_kernel<C, TIn>, smem, done);
+    cudaError_t e = ensure_smem(sar_rcmc_filter_ifft_kernel<C, TIn, SLAB>, smem, done);
     if (e != cudaSuccess) return e;
-    sar_rcmc_filter_ifft_kernel<C, TIn><<<(unsigned)a.tiles, C::THREADS, smem, st>>>(a);
+    sar_rcmc_filter_ifft_kernel<C, TIn, SLAB><<<(unsigned)a.tiles, C::THREADS, smem, st>>>(a);
+    g_launch_count.fetch_add(1, std::memory_order_relaxed);
+    return cudaGetLastError();
+}
+template <class T>
+cudaError_t launch_rcmc_slab(const SarArgs& a, cudaStream_t st) {
+    using L = RcmcSlab<T, T>;
+    const unsigned grid = (unsigned)((a.na / L::ROWS) * (a.nr / L::NC));
+    sar_rcmc_filter_slab_kernel<T, T><<<grid, L::THREADS, 0, st>>>(a);
     g_launch_count.fetch_add(1, std::memory_order_relaxed);
     return cudaGetLastError();
 }
 
 struct SarEntry {
     int n, dtype, w, tw_total;
+    bool slab;
     cudaError_t (*launch)(const SarArgs&, cudaStream_t);
     cudaError_t (*build_tw)(float2*, cudaStream_t);
 };
-template <class C, class T, bool RANGE>
+template <class C, class T, bool RANGE, bool SLAB>
 constexpr SarEntry sar_entry() {
-    if constexpr (RANGE) return SarEntry{C::N, T::ELEM_BYTES == 8 ? 0 : 1, C::W, C::TW_TOTAL, &launch_range<C, T>, &launch_build_tw<C>};
-    else return SarEntry{C::N, T::ELEM_BYTES == 8 ? 0 : 1, C::W, C::TW_TOTAL, &launch_rcmc<C, T>, &launch_build_tw<C>};
+    if constexpr (RANGE)
+        return SarEntry{C::N, T::ELEM_BYTES == 8 ? 0 : 1, C::W, C::TW_TOTAL, SLAB, &launch_range<C, T, SLAB>, &launch_build_tw<C>};
+    else
+        return SarEntry{C::N, T::ELEM_BYTES == 8 ? 0 : 1, C::W, C::TW_TOTAL, SLAB, &launch_rcmc<C, T, SLAB>, &launch_build_tw<C>};
 }
-#define SAR_PAIR(C, RANGE) sar_entry<C, StoreC64, RANGE>(), sar_entry<C, StoreC32H, RANGE>()
-static const SarEntry k_range[] = {SAR_PAIR(R1024p, true), SAR_PAIR(R2048, true), SAR_PAIR(R4096, true), SAR_PAIR(R8192, true)};
-static const SarEntry k_rcmc[] = {SAR_PAIR(T1024, false), SAR_PAIR(T2048, false), SAR_PAIR(T4096, false)};
+#define SAR_QUAD(C, RANGE)                                                                        \
+    sar_entry<C, StoreC64, RANGE, false>(), sar_entry<C, StoreC32H, RANGE, false>(),             \
+    sar_entry<C, StoreC64, RANGE, true>(), sar_entry<C, StoreC32H, RANGE, true>()
+static const SarEntry k_range[] = {SAR_QUAD(R1024p, true), SAR_QUAD(R2048, true), SAR_QUAD(R4096, true), SAR_QUAD(R8192, true)};
+static const SarEntry k_rcmc[] = {SAR_QUAD(T1024, false), SAR_QUAD(T2048, false), SAR_QUAD(T4096, false)};
 
 template <size_t K>
-static const SarEntry* find(const SarEntry (&tab)[K], int n, int dtype) {
+static const SarEntry* find(const SarEntry (&tab)[K], int n, int dtype, bool slab) {
     for (const SarEntry& e : tab)
-        if (e.n == n && e.dtype == dtype) return &e;
+        if (e.n == n && e.dtype == dtype && e.slab == slab) return &e;
     return nullptr;
+}
+
+// largest spread of the integer shift inside one CTA of the slab row pass (32 Doppler bins x NC range
+// bins), over the whole image, in float64
+static double slab_shift_spread(const sar_rda_desc* d, int nc) {
+    const double wavelength = kLight / d->carrier_hz, dr = kLight / (2.0 * d->fs_hz);
+    const int na = (int)d->n_azimuth, nr = (int)d->n_range;
+    auto mig = [&](int k, int n) {
+        const int kk = (k < na / 2) ? k : k - na;
+        const double f = (double)kk * d->prf_hz / (double)na;
+        const double aa = wavelength * f / (2.0 * d->velocity_mps), u = aa * aa, sq = sqrt(1.0 - u);
+        return (d->r_center_m / dr - (double)(nr / 2) + (double)n) * (u / ((1.0 + sq) * sq));
+    };
+    double worst = 0.0;
+    for (int k0 = 0; k0 + 31 < na; k0 += 32) {
+        // the spread is largest at the far end of the swath
+        const double lo = fmin(mig(k0, nr - nc), mig(k0 + 31, nr - nc));
+        const double hi = fmax(mig(k0, nr - 1), mig(k0 + 31, nr - 1));
+        worst = fmax(worst, hi - lo);
+    }
+    return worst;
 }
 
 }  // namespace b200fft
@@ -479,12 +657,21 @@ using namespace b200fft;
 
 struct b200fft_sar_s {
     sar_rda_desc d;
+    // row-major intermediate ("layout" 0)
     const SarEntry* range;
     const KernelEntry* azfft;
     const SarEntry* rcmc;
     const KernelEntry* azifft;   // in-place inverse column transform of the unfused variant
-    bool fused;                  // step 2 as one kernel (true) or as row pass + column pass (false)
     bool can_unfuse;
+    // slab intermediate ("layout" 1)
+    const SarEntry* range_slab;
+    const SarEntry* rcmc_slab;
+    const KernelEntry* azfft_slab[2];    // forward column tiles of 2 and of 4 range bins, intermediate type both ways
+    const KernelEntry* azifft_slab[2];   // inverse column tiles, intermediate type in, complex64 out
+    bool can_slab;
+    int layout;                  // 0 row-major, 1 slab
+    int tile_columns;            // slab layout: range bins per column tile, 2 or 4
+    bool fused;                  // step 2 as one kernel (true) or as row pass + column pass (false)
     float2 *tw_range, *tw_az, *H;
     float4 *mig, *phs;
     float2* stp;
@@ -499,6 +686,10 @@ static void sar_release(b200fft_sar_s* p) {
     if (p->mig) cudaFree(p->mig);
     if (p->phs) cudaFree(p->phs);
     if (p->stp) cudaFree(p->stp);
+}
+
+static size_t image_bytes(const b200fft_sar_s* p) {
+    return (size_t)p->d.n_azimuth * (size_t)p->d.n_range * (p->d.intermediate_dtype == B200FFT_C64 ? 8 : 4);
 }
 
 extern "C" int sar_rda_params_create(sar_rda_params_t* params, const sar_rda_desc* d) {
@@ -522,29 +713,50 @@ extern "C" int sar_rda_params_create(sar_rda_params_t* params, const sar_rda_des
     if (!p) return B200FFT_ERR_ALLOC;
     p->d = *d;
     const int na = (int)d->n_azimuth, nr = (int)d->n_range, dt = d->intermediate_dtype;
-    p->range = find(k_range, nr, dt);
+    p->range = find(k_range, nr, dt, false);
+    p->range_slab = find(k_range, nr, dt, true);
     // Column tiles. With fp16 intermediates the wider tile on a cluster of two CTAs (32-byte instead of 16-byte
     // row segments at n_azimuth = 4096: 84 -> 77 us); with complex64 the 4-column tile measured faster inside the
     // chain (85 against 88 us per pass), where part of the image still sits in L2.
     auto cols_kernel = [&](bool inverse, int dtype) {
         if (dtype == B200FFT_C32H) {
-            const KernelEntry* k = find_cols_kernel(na, inverse, dtype, dtype, 1023);
+            const KernelEntry* k = find_cols_kernel(na, inverse, dtype, dtype, 0, VAR_WIDE_CLUSTER);
             if (k && nr % k->w == 0) return k;
         }
         return find_cols_kernel(na, inverse, dtype, dtype, 1);
     };
     p->azfft = cols_kernel(false, dt);
-    p->rcmc = find(k_rcmc, na, dt);
+    p->rcmc = find(k_rcmc, na, dt, false);
+    p->rcmc_slab = find(k_rcmc, na, dt, true);
     p->azifft = cols_kernel(true, B200FFT_C64);
+    for (int i = 0; i < 2; ++i) {
+        p->azfft_slab[i] = find_sar_cols_kernel(na, 2 << i, false, dt, dt);
+        p->azifft_slab[i] = find_sar_cols_kernel(na, 2 << i, true, dt, B200FFT_C64);
+    }
     {   // the row pass stages COLS + HALO samples: the shift may grow by at most HALO - 16 bins over COLS bins
         const double aa = wavelength * d->prf_hz / (4.0 * d->velocity_mps), u = aa * aa, sq = sqrt(1.0 - u);
         const double gmax = u / ((1.0 + sq) * sq);
         p->can_unfuse = p->azifft != nullptr && nr % RcmcRows::COLS == 0 &&
                         gmax * RcmcRows::COLS + 16.0 <= (double)RcmcRows::HALO;
-        p->fused = !p->can_unfuse;
     }
+    using RS = RcmcSlab<StoreC64, StoreC64>;
+    p->can_slab = p->range_slab && p->rcmc_slab && p->azfft_slab[0] && p->azfft_slab[1] && p->azifft_slab[0] &&
+                  p->azifft_slab[1] && na % 64 == 0 && nr % RS::NC == 0 &&
+                  slab_shift_spread(d, RS::NC) + 2.0 <= (double)RS::MAX_SPREAD;
+    p->layout = p->can_slab ? 1 : 0;
+    p->tile_columns = 2;
+    p->fused = p->layout == 0 && !p->can_unfuse;
     if (!p->range || !p->azfft || !p->rcmc || d->n_azimuth > 16384 || d->n_range > 16384 || nr % p->rcmc->w) {
         delete p;
+        return B200FFT_ERR_UNSUPPORTED;
+    }
+    static_assert(T1024::TW_TOTAL == S1024::TW_TOTAL && T2048::TW_TOTAL == S2048::TW_TOTAL && T4096::TW_TOTAL == S4096::TW_TOTAL &&
+                      T4096::radix(1) == S4096::radix(1) && T4096::radix(2) == S4096::radix(2) &&
+                      T2048::radix(1) == S2048::radix(1) && T2048::radix(2) == S2048::radix(2) &&
+                      T1024::radix(1) == S1024::radix(1) && T1024::radix(2) == S1024::radix(2),
+                  "the 2- and 4-column tiles share one twiddle table: same factorisation");
+    if (p->azfft->tw_total != p->rcmc->tw_total || (p->azifft && p->azifft->tw_total != p->rcmc->tw_total)) {
+        delete p;                  // every azimuth kernel reads the one table built below
         return B200FFT_ERR_UNSUPPORTED;
     }
     bool ok = cudaMalloc(&p->tw_range, sizeof(float2) * (size_t)p->range->tw_total) == cudaSuccess &&
@@ -578,7 +790,7 @@ extern "C" int sar_rda_params_create(sar_rda_params_t* params, const sar_rda_des
 
 extern "C" int sar_rda_workspace_bytes(sar_rda_params_t p, size_t* bytes) {
     if (!p || !bytes) return B200FFT_ERR_INVALID_ARG;
-    *bytes = (size_t)p->d.n_azimuth * (size_t)p->d.n_range * (p->d.intermediate_dtype == B200FFT_C64 ? 8 : 4);
+    *bytes = 2 * image_bytes(p);       // two intermediate images (the slab layout's step 2 goes from one to the other)
     return B200FFT_OK;
 }
 
@@ -598,50 +810,87 @@ extern "C" int sar_rda_run_step(const void* raw, sar_rda_params_t p, void* out, 
     if (!p->workspace) return B200FFT_ERR_WORKSPACE;
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
     const int64_t na = p->d.n_azimuth, nr = p->d.n_range;
+    const bool slab = p->layout == 1;
+    const int dt = p->d.intermediate_dtype;
+    const int gcols = dt == B200FFT_C64 ? 4 : 8;                 // range bins per 32-byte granule
+    void* buf0 = p->workspace;
+    void* buf1 = static_cast<char*>(p->workspace) + image_bytes(p);
+    auto ok = [](cudaError_t e) { return e == cudaSuccess ? B200FFT_OK : B200FFT_ERR_CUDA; };
+    auto slab_geometry = [&](FftArgs& f, int w) {
+        f.tpg = gcols / w;
+        f.slab_stride = na * gcols;
+        f.dist = gcols;
+    };
     if (step == 0) {
         if (!raw) return B200FFT_ERR_INVALID_ARG;
         if (reinterpret_cast<uintptr_t>(raw) % 16) return B200FFT_ERR_ALIGNMENT;
         SarArgs a{};
-        a.in = raw; a.out = p->workspace; a.tw = p->tw_range;
+        a.in = raw; a.out = buf0; a.tw = p->tw_range;
         a.tab = SarTables{p->H, p->mig, p->phs, p->stp};
-        a.tiles = na; a.ld = nr; a.nr = (int)nr; a.scale = 1.0f;
-        return p->range->launch(a, st) == cudaSuccess ? B200FFT_OK : B200FFT_ERR_CUDA;
+        a.tiles = na; a.ld = nr; a.nr = (int)nr; a.na = (int)na; a.scale = 1.0f;
+        return ok((slab ? p->range_slab : p->range)->launch(a, st));
     }
     if (step == 1) {
         FftArgs a{};
-        a.in = p->workspace; a.out = p->workspace; a.tw = p->tw_az;
-        a.tiles = nr / p->azfft->w; a.dist = nr;
+        a.in = buf0; a.out = buf0; a.tw = p->tw_az;
         a.scale = (float)(1.0 / (double)na);
         a.prefetch_ahead = 0;
-        return p->azfft->launch(a, st) == cudaSuccess ? B200FFT_OK : B200FFT_ERR_CUDA;
+        const KernelEntry* k = slab ? p->azfft_slab[p->tile_columns == 4] : p->azfft;
+        a.tiles = nr / k->w; a.dist = nr;
+        if (slab) slab_geometry(a, k->w);
+        return ok(k->launch(a, st));
     }
     if (!out) return B200FFT_ERR_INVALID_ARG;
     if (reinterpret_cast<uintptr_t>(out) % 16) return B200FFT_ERR_ALIGNMENT;
     SarArgs a{};
-    a.in = p->workspace; a.out = out; a.tw = p->tw_az;
+    a.in = buf0; a.out = out; a.tw = p->tw_az;
     a.tab = SarTables{p->H, p->mig, p->phs, p->stp};
-    a.tiles = nr / p->rcmc->w; a.ld = nr; a.nr = (int)nr; a.scale = 1.0f;
-    if (p->fused) return p->rcmc->launch(a, st) == cudaSuccess ? B200FFT_OK : B200FFT_ERR_CUDA;
+    a.tiles = nr / p->rcmc->w; a.ld = nr; a.nr = (int)nr; a.na = (int)na; a.scale = 1.0f;
+    if (p->fused) return ok((slab ? p->rcmc_slab : p->rcmc)->launch(a, st));
+    FftArgs f{};
+    f.tw = p->tw_az;
+    f.scale = 1.0f;                         // 1/n_azimuth was applied after the forward azimuth FFT
+    f.prefetch_ahead = 0;
+    if (slab) {
+        a.out = buf1;
+        cudaError_t e = dt == B200FFT_C64 ? launch_rcmc_slab<StoreC64>(a, st) : launch_rcmc_slab<StoreC32H>(a, st);
+        if (e != cudaSuccess) return B200FFT_ERR_CUDA;
+        const KernelEntry* k = p->azifft_slab[p->tile_columns == 4];
+        f.in = buf1; f.out = out;
+        f.tiles = nr / k->w;
+        slab_geometry(f, k->w);
+        f.out_dist = nr;                    // the image leaves row-major
+        return ok(k->launch(f, st));
+    }
     const int chunks = (int)(nr / RcmcRows::COLS);
-    if (p->d.intermediate_dtype == B200FFT_C64)
+    if (dt == B200FFT_C64)
         sar_rcmc_filter_rows_kernel<StoreC64><<<(unsigned)(na * chunks), RcmcRows::TPB, 0, st>>>(a, chunks);
     else
         sar_rcmc_filter_rows_kernel<StoreC32H><<<(unsigned)(na * chunks), RcmcRows::TPB, 0, st>>>(a, chunks);
     g_launch_count.fetch_add(1, std::memory_order_relaxed);
     if (cudaGetLastError() != cudaSuccess) return B200FFT_ERR_CUDA;
-    FftArgs f{};
-    f.in = out; f.out = out; f.tw = p->tw_az;
+    f.in = out; f.out = out;
     f.tiles = nr / p->azifft->w; f.dist = nr;
-    f.scale = 1.0f;                         // 1/n_azimuth was applied after the forward azimuth FFT
-    f.prefetch_ahead = 0;
-    return p->azifft->launch(f, st) == cudaSuccess ? B200FFT_OK : B200FFT_ERR_CUDA;
+    return ok(p->azifft->launch(f, st));
 }
 
 extern "C" int sar_rda_set_option(sar_rda_params_t p, const char* key, int64_t value) {
     if (!p || !key) return B200FFT_ERR_INVALID_ARG;
     if (std::strcmp(key, "fused_rcmc") == 0) {
-        if (!value && !p->can_unfuse) return B200FFT_ERR_UNSUPPORTED;
+        if (!value && p->layout == 0 && !p->can_unfuse) return B200FFT_ERR_UNSUPPORTED;
         p->fused = value != 0;
+        return B200FFT_OK;
+    }
+    if (std::strcmp(key, "layout") == 0) {
+        if (value != 0 && value != 1) return B200FFT_ERR_INVALID_ARG;
+        if (value == 1 && !p->can_slab) return B200FFT_ERR_UNSUPPORTED;
+        p->layout = (int)value;
+        if (value == 0 && !p->can_unfuse) p->fused = true;
+        return B200FFT_OK;
+    }
+    if (std::strcmp(key, "tile_columns") == 0) {
+        if (value != 2 && value != 4) return B200FFT_ERR_INVALID_ARG;
+        p->tile_columns = (int)value;
         return B200FFT_OK;
     }
     return B200FFT_ERR_INVALID_ARG;

@@ -19,25 +19,43 @@ def _need_gpu():
         pytest.skip("no CUDA device")
 
 
-def _gpu_chain(scene, raw, dtype, steps=False, fused=None):
+def _gpu_chain(scene, raw, dtype, steps=False, fused=None, layout=None, tile_columns=None):
+    """Run the chain through the C ABI. layout: 0 = row-major intermediates, 1 = slab layout (the
+    default); tile_columns: range bins per column tile on the slab layout."""
     import torch
     from paper_2609_32237_b200 import binding as B
     p = B.sar_rda_params_create(B.sar_desc_from_scene(scene, dtype))
     try:
+        if layout is not None:
+            B.sar_rda_set_option(p, "layout", int(layout))
+        if tile_columns is not None:
+            B.sar_rda_set_option(p, "tile_columns", int(tile_columns))
         if fused is not None:
             B.sar_rda_set_option(p, "fused_rcmc", int(fused))
         need = B.sar_rda_workspace_bytes(p)
-        assert need == scene.n_azimuth * scene.n_range * (8 if dtype == C64 else 4)
+        na, nr = scene.n_azimuth, scene.n_range
+        image = na * nr * (8 if dtype == C64 else 4)
+        assert need == 2 * image
         ws = torch.zeros(need, dtype=torch.uint8, device="cuda")
         B.sar_rda_set_workspace(p, ws.data_ptr(), need)
         rd = to_device_c64(raw)
         out = torch.zeros_like(rd)
         st = torch.cuda.current_stream().cuda_stream
+        slab = layout is None or layout == 1
 
         def ws_as_complex():
+            """The first intermediate image as a row-major complex128 matrix (undoing the slab
+            layout: granules of 32 bytes, element (k, n) at ((n // G) * na + k) * G + n % G)."""
+            first = ws[:image]
             if dtype == C64:
-                return ws.view(torch.complex64).reshape(scene.n_azimuth, scene.n_range).cpu().numpy().astype(np.complex128)
-            return half_to_c128(ws.view(torch.float16).reshape(scene.n_azimuth, scene.n_range, 2))
+                a = first.view(torch.complex64).cpu().numpy().astype(np.complex128)
+                g = 4
+            else:
+                a = half_to_c128(first.view(torch.float16).reshape(-1, 2))
+                g = 8
+            if slab:
+                return a.reshape(nr // g, na, g).transpose(1, 0, 2).reshape(na, nr)
+            return a.reshape(na, nr)
 
         if steps:
             inter = []
@@ -69,9 +87,13 @@ def small_scene():
     return sc, raw, rc, S, img
 
 
-def test_small_scene_each_pass_fp32(small_scene):
+LAYOUTS = [(0, None), (1, 2), (1, 4)]          # (layout, tile_columns)
+
+
+@pytest.mark.parametrize("layout,tile_columns", LAYOUTS)
+def test_small_scene_each_pass_fp32(small_scene, layout, tile_columns):
     sc, raw, rc, S, img = small_scene
-    got, inter = _gpu_chain(sc, raw, C64, steps=True)
+    got, inter = _gpu_chain(sc, raw, C64, steps=True, layout=layout, tile_columns=tile_columns)
     assert rel_l2(inter[0], rc) <= 1e-5                      # fused range compression
     assert rel_l2(inter[1], S / sc.n_azimuth) <= 1e-5        # azimuth FFT, scaled 1/N_a
     assert rel_l2(got, img) <= 1e-5
@@ -79,9 +101,10 @@ def test_small_scene_each_pass_fp32(small_scene):
         assert quality.peak_cell(got, tuple(cell)) == tuple(cell)
 
 
-def test_small_scene_fp16_intermediates(small_scene):
+@pytest.mark.parametrize("layout,tile_columns", LAYOUTS)
+def test_small_scene_fp16_intermediates(small_scene, layout, tile_columns):
     sc, raw, rc, S, img = small_scene
-    got, inter = _gpu_chain(sc, raw, C32H, steps=True)
+    got, inter = _gpu_chain(sc, raw, C32H, steps=True, layout=layout, tile_columns=tile_columns)
     assert rel_l2(inter[0], rc) <= 5e-3
     assert rel_l2(inter[1], S / sc.n_azimuth) <= 5e-3
     assert rel_l2(got, img) <= 5e-3
@@ -89,15 +112,17 @@ def test_small_scene_fp16_intermediates(small_scene):
         assert quality.peak_cell(got, tuple(cell)) == tuple(cell)
 
 
+@pytest.mark.parametrize("layout", [0, 1])
 @pytest.mark.parametrize("dtype,tol", [(C64, 1e-5), (C32H, 5e-3)])
-def test_small_scene_fused_and_unfused_step2_agree(small_scene, dtype, tol):
-    """Step 2 as one fused kernel and as row pass + in-place column pass: both within
-    tolerance of the oracle, and equal to each other to rounding."""
+def test_small_scene_fused_and_unfused_step2_agree(small_scene, dtype, tol, layout):
+    """Step 2 as one fused kernel and as row pass + column pass: both within tolerance of the
+    oracle, and equal to each other to rounding (with fp16 intermediates the slab layout's row
+    pass rounds once more to fp16, which the fused kernel does not)."""
     sc, raw, rc, S, img = small_scene
-    a = _gpu_chain(sc, raw, dtype, fused=True)
-    b = _gpu_chain(sc, raw, dtype, fused=False)
+    a = _gpu_chain(sc, raw, dtype, fused=True, layout=layout)
+    b = _gpu_chain(sc, raw, dtype, fused=False, layout=layout)
     assert rel_l2(a, img) <= tol and rel_l2(b, img) <= tol
-    assert rel_l2(a, b) <= 2e-6
+    assert rel_l2(a, b) <= (2e-6 if (dtype == C64 or layout == 0) else 1e-3)
     for cell in sc.targets:
         assert quality.peak_cell(a, tuple(cell)) == tuple(cell)
         assert quality.peak_cell(b, tuple(cell)) == tuple(cell)
@@ -115,13 +140,14 @@ def test_single_on_grid_echo_compresses_to_the_pulse_length():
     assert np.abs(inter[0][6]).max() == 0
 
 
+@pytest.mark.parametrize("layout,tile_columns", LAYOUTS)
 @pytest.mark.parametrize("fused", [False, True])
 @pytest.mark.parametrize("dtype,tol", [(C64, 1e-5), (C32H, 5e-3)])
-def test_config4_full_scene(dtype, tol, fused, full_scene):
+def test_config4_full_scene(dtype, tol, fused, layout, tile_columns, full_scene):
     """4096 x 4096, 16 seeded unit targets, noise at 20 dB: whole image and peak cells,
-    for both forms of step 2."""
+    for both forms of step 2 and both intermediate layouts."""
     sc, raw, img = full_scene
-    got = _gpu_chain(sc, raw, dtype, fused=fused)
+    got = _gpu_chain(sc, raw, dtype, fused=fused, layout=layout, tile_columns=tile_columns)
     err = rel_l2(got, img)
     assert err <= tol, err
     for cell in sc.targets:
@@ -149,11 +175,12 @@ def l_band_case():
     return sc, raw, img
 
 
+@pytest.mark.parametrize("layout", [0, 1])
 @pytest.mark.parametrize("fused", [False, True])
 @pytest.mark.parametrize("dtype,tol", [(C64, 1e-5), (C32H, 5e-3)])
-def test_l_band_scene_with_large_shifts(dtype, tol, fused, l_band_case):
+def test_l_band_scene_with_large_shifts(dtype, tol, fused, layout, l_band_case):
     sc, raw, img = l_band_case
-    got = _gpu_chain(sc, raw, dtype, fused=fused)
+    got = _gpu_chain(sc, raw, dtype, fused=fused, layout=layout)
     err = rel_l2(got, img)
     assert err <= tol, err
     for cell in sc.targets:
@@ -182,8 +209,8 @@ def test_other_frame_sizes_and_error_paths():
     raw = inputs.simulate_raw(sc, seed=11)
     img = oracle.sar_rda(oracle.sar_params(sc), raw)
     for dtype, tol in ((C64, 1e-5), (C32H, 5e-3)):
-        for fused in (False, True):
-            got = _gpu_chain(sc, raw, dtype, fused=fused)
+        for fused, layout in ((False, 0), (True, 0), (False, 1), (True, 1)):
+            got = _gpu_chain(sc, raw, dtype, fused=fused, layout=layout)
             assert rel_l2(got, img) <= tol
             for cell in sc.targets:
                 assert quality.peak_cell(got, tuple(cell)) == tuple(cell)
@@ -195,7 +222,7 @@ def test_other_frame_sizes_and_error_paths():
             B.sar_rda_form_image(rd.data_ptr(), p, out.data_ptr(), 0)
         assert e.value.status == 6
         need = B.sar_rda_workspace_bytes(p)
-        small = torch.zeros(need // 2, dtype=torch.uint8, device="cuda")
+        small = torch.zeros(need // 2, dtype=torch.uint8, device="cuda")   # one image instead of two
         with pytest.raises(B.B200FftError) as e:
             B.sar_rda_set_workspace(p, small.data_ptr(), need // 2)
         assert e.value.status == 6
