@@ -18,27 +18,28 @@ namespace b200fft {
 // plain loads. After the last stage the results go back to shared memory as a dense image (the exchange
 // buffer is free by then) and leave as TMA stores, which the next tile's first stage overlaps; the stores
 // must have read shared memory before the next exchange overwrites it (wait_group.read). Tensor maps cover
-// this GPU's own memory; no multicast. Every wait is bounded: a CTA whose wait runs out raises
+// this GPU's own memory; no multicast. (Two-column tiles at two CTAs per multiprocessor, i.e. boxes with
+// 16-byte rows, measured twice as slow: 144 against 74 us on 4096 x 4096.) Every wait is bounded: a CTA whose wait runs out raises
 // g_tma_timeouts once, stops taking tiles, waits (bounded again) for the copies it still has in flight
 // and returns; the output of that call is then incomplete.
 __device__ int g_tma_timeouts = 0;   // CTAs whose wait for a copy ran out of polls (never expected)
 
-template <class C, class TIn>
+template <class C, class TIn, int CPS = 1>     // CPS: CTAs per multiprocessor the shared memory is divided among
 struct Stream {
     static constexpr int BOX_ROWS = 256, NBOX = C::N / BOX_ROWS;
     static constexpr int X_BYTES = C::N * C::W * 8;                         // exchange buffer = output image
     static constexpr int BOX_BYTES = BOX_ROWS * C::W * TIn::ELEM_BYTES;
-    static constexpr int ROOM = 232448 - 2048 - X_BYTES;
+    static constexpr int ROOM = 232448 / CPS - 2048 - X_BYTES;
     static constexpr int SBOX = (ROOM / BOX_BYTES) < NBOX ? (ROOM / BOX_BYTES) : NBOX;   // boxes staged by TMA
     static constexpr int SMEM_BYTES = X_BYTES + SBOX * BOX_BYTES;
     static_assert(C::N % BOX_ROWS == 0 && SBOX >= 1, "whole boxes");
     static_assert(C::CL == 1 && C::G == 1 && C::W >= 2 && C::THREADS >= NBOX, "single-CTA column tiles");
 };
 
-template <class C, bool INV, class TIn, class TOut>
-__global__ void __launch_bounds__(C::THREADS, 1)
+template <class C, bool INV, class TIn, class TOut, int CPS>
+__global__ void __launch_bounds__(C::THREADS, CPS)
     fft_cols_stream_kernel(const FftArgs a, const __grid_constant__ CUtensorMap tm_in, const __grid_constant__ CUtensorMap tm_out) {
-    using L = Stream<C, TIn>;
+    using L = Stream<C, TIn, CPS>;
     extern __shared__ __align__(128) float2 smem_stream[];   // TMA destinations and sources are 128-byte aligned
     constexpr int W = C::W, N = C::N, S = C::S;
     constexpr int XW_IN = W * TIn::ELEM_BYTES / 4, XW_OUT = W * TOut::ELEM_BYTES / 4;   // tile width in 4-byte map elements
@@ -179,12 +180,12 @@ static bool make_column_map(CUtensorMap* m, const void* base, int64_t rows, int6
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <class C, bool INV, class TI, class TO>
+template <class C, bool INV, class TI, class TO, int CPS>
 cudaError_t launch_cols_stream(const FftArgs& a, cudaStream_t st) {
-    using L = Stream<C, TI>;
+    using L = Stream<C, TI, CPS>;
     static bool done[64] = {};
     static int sms[64] = {};
-    cudaError_t e = ensure_smem(fft_cols_stream_kernel<C, INV, TI, TO>, L::SMEM_BYTES, done);
+    cudaError_t e = ensure_smem(fft_cols_stream_kernel<C, INV, TI, TO, CPS>, L::SMEM_BYTES, done);
     if (e != cudaSuccess) return e;
     // the copy engine wants 16-byte aligned bases and row pitches, and tile columns that start on 16 bytes
     if ((reinterpret_cast<uintptr_t>(a.in) & 15) || (reinterpret_cast<uintptr_t>(a.out) & 15) ||
@@ -198,16 +199,18 @@ cudaError_t launch_cols_stream(const FftArgs& a, cudaStream_t st) {
     cudaGetDevice(&dev);
     if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
     if (!sms[dev]) cudaDeviceGetAttribute(&sms[dev], cudaDevAttrMultiProcessorCount, dev);
-    const unsigned grid = (unsigned)(a.tiles < sms[dev] ? a.tiles : sms[dev]);
-    fft_cols_stream_kernel<C, INV, TI, TO><<<grid, C::THREADS, L::SMEM_BYTES, st>>>(a, tin, tout);
+    const int64_t slots = (int64_t)sms[dev] * CPS;
+    const unsigned grid = (unsigned)(a.tiles < slots ? a.tiles : slots);
+    fft_cols_stream_kernel<C, INV, TI, TO, CPS><<<grid, C::THREADS, L::SMEM_BYTES, st>>>(a, tin, tout);
     g_launch_count.fetch_add(1, std::memory_order_relaxed);
     return cudaGetLastError();
 }
-template <class C, bool INV, class TS>
+template <class C, bool INV, class TS, int CPS = 1>
 constexpr KernelEntry make_stream_entry() {
-    return KernelEntry{C::N, C::W, C::G, 1, C::THREADS, Stream<C, TS>::SMEM_BYTES, C::TW_TOTAL, VAR_STREAM, INV,
+    return KernelEntry{C::N, C::W, C::G, 1, C::THREADS, Stream<C, TS, CPS>::SMEM_BYTES, C::TW_TOTAL,
+                       VAR_STREAM, INV,
                        TS::ELEM_BYTES == 8 ? 0 : 1, TS::ELEM_BYTES == 8 ? 0 : 1,
-                       &launch_cols_stream<C, INV, TS, TS>, &launch_build_tw<C>};
+                       &launch_cols_stream<C, INV, TS, TS, CPS>, &launch_build_tw<C>};
 }
 static const KernelEntry k_cols_stream[] = {
     make_stream_entry<T4096, false, StoreC64>(), make_stream_entry<T4096, true, StoreC64>(),

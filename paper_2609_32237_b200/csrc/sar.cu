@@ -399,26 +399,53 @@ __global__ void __launch_bounds__(RcmcRows::TPB) sar_rcmc_filter_rows_kernel(con
 }
 
 // ---------------------------------------------------------------- step 2a on the slab layout
-// Range cell migration correction and azimuth filter, slab image to slab image. A CTA works on 32
-// consecutive Doppler bins (the lanes of every warp) by NC consecutive range bins (four per thread);
-// in the slab layout the 32 rows of one granule column are one contiguous kilobyte, so the window
-// is staged with whole-line loads, the results leave as whole lines, and a lane's taps sit in its
-// own shared-memory column (conflict-free whatever the row's shift is). The window of every CTA
-// starts at its smallest integer shift; how far the shift may spread inside a CTA is checked when
-// the parameters are created.
+// The same row pass for the slab layout, organised the other way round. A CTA works on 32 consecutive
+// Doppler bins (the lanes of every warp) by NC consecutive range bins (four per thread). The window of samples it needs is staged in shared memory as [sample][row] with an
+// odd pitch, so a lane's eight taps come from its own column: conflict-free whatever the row's shift is.
+// The four pixels of a thread share one window of 11 samples when their integer shifts agree (else each
+// fetches its own eight). The window of a CTA starts at its smallest integer shift; how far the shift may
+// spread inside a CTA is checked when the parameters are created. In the slab layout 32 rows of a granule
+// column are one contiguous kilobyte, so the window arrives and the results leave as whole lines. (The same
+// organisation on row-major images, with the results turned around in shared memory before they are
+// stored, measured 140 us against 89 us for the row-wise kernel above: its loads are exposed with two CTAs
+// per multiprocessor; it was dropped.)
 template <class TIn, class TOut>
-struct RcmcSlab {
-    static constexpr int ROWS = 32, NC = 64, HALO = 32, NS = NC + HALO;
+struct RcmcPass {
+    static constexpr int ROWS = 32, NC = 64, HALO = 32, NS = NC + HALO, PITCH = ROWS + 1;
     static constexpr int THREADS = NC / 4 * 32;
     static constexpr int GI = 32 / TIn::ELEM_BYTES, GO = 32 / TOut::ELEM_BYTES;
     static constexpr int MAX_SPREAD = HALO - 8 - 6;     // allowed (largest - smallest) integer shift in a CTA
 };
 
+// interpolator weights of two pixels at once (lane x: first pixel, lane y: second), as magnitudes with the
+// sign (-1)^j left to the caller like sinc8_weights_rcp. The eight reciprocals 1 / (mu - j) come two at a
+// time from one hardware reciprocal of their product (1/a = b / (ab)), and the sums and products run as
+// packed fp32 pairs: about 22 issue slots and 5 special-function operations per pixel.
+__device__ __forceinline__ void sinc8_weights_pair(float mua, float mub, float2 (&w)[8]) {
+    const float2 mu = make_float2(fmaxf(mua, 1e-30f), fmaxf(mub, 1e-30f));
+    float2 x[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) x[i] = (i == 3) ? mu : __fadd2_rn(mu, make_float2((float)(3 - i), (float)(3 - i)));
+#pragma unroll
+    for (int h = 0; h < 4; ++h) {
+        const float2 pr = __fmul2_rn(x[2 * h], x[2 * h + 1]);
+        const float2 r = make_float2(rcp_approx(pr.x), rcp_approx(pr.y));
+        w[2 * h] = __fmul2_rn(x[2 * h + 1], r);
+        w[2 * h + 1] = __fmul2_rn(x[2 * h], r);
+    }
+    float2 s = make_float2(0.f, 0.f);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) s = ((i - 3) & 1) ? s - w[i] : s + w[i];
+    const float2 inv = make_float2(rcp_approx(s.x), rcp_approx(s.y));
+#pragma unroll
+    for (int i = 0; i < 8; ++i) w[i] = __fmul2_rn(w[i], inv);
+}
+
 template <class TIn, class TOut>
-__global__ void __launch_bounds__(RcmcSlab<TIn, TOut>::THREADS) sar_rcmc_filter_slab_kernel(const SarArgs a) {
-    using L = RcmcSlab<TIn, TOut>;
-    constexpr int NS = L::NS, GI = L::GI, GO = L::GO;
-    __shared__ __align__(16) float2 win[NS * 32];       // [sample][row]
+__global__ void __launch_bounds__(RcmcPass<TIn, TOut>::THREADS) sar_rcmc_filter_slab_kernel(const SarArgs a) {
+    using L = RcmcPass<TIn, TOut>;
+    constexpr int NS = L::NS, GI = L::GI, GO = L::GO, PITCH = L::PITCH, EBI = TIn::ELEM_BYTES;
+    __shared__ __align__(16) float2 win[NS * PITCH];     // [sample][row]
     const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
     const int kblocks = a.na / 32;
     const int k0 = (blockIdx.x % kblocks) * 32, n0 = (blockIdx.x / kblocks) * L::NC;
@@ -433,26 +460,32 @@ __global__ void __launch_bounds__(RcmcSlab<TIn, TOut>::THREADS) sar_rcmc_filter_
         migration(__ldg(a.tab.mig + k0 + 31), n0, ib, mu);
         s0 = (n0 + min(ia, ib) - 3) & ~(GI - 1);        // floors for negative values too
     }
-    {   // stage the window: 16-byte pieces, a warp takes one half of the granules of 32 rows
-        const char* in = reinterpret_cast<const char*>(a.in);
+    auto put = [&](float2* dst, const uint4 v) {         // 16 bytes = GRAN samples, converted to fp32
+        if constexpr (EBI == 8) {
+            dst[0] = make_float2(__uint_as_float(v.x), __uint_as_float(v.y));
+            dst[PITCH] = make_float2(__uint_as_float(v.z), __uint_as_float(v.w));
+        } else {
+            dst[0] = __half22float2(*reinterpret_cast<const __half2*>(&v.x));
+            dst[PITCH] = __half22float2(*reinterpret_cast<const __half2*>(&v.y));
+            dst[2 * PITCH] = __half22float2(*reinterpret_cast<const __half2*>(&v.z));
+            dst[3 * PITCH] = __half22float2(*reinterpret_cast<const __half2*>(&v.w));
+        }
+    };
+    const char* in = reinterpret_cast<const char*>(a.in);
+    {   // a warp takes one half of the granules of 32 rows at a time: lanes = rows
         const int slab0 = s0 / GI;                       // exact: s0 is a multiple of GI
         const int nslabs = a.nr / GI;
-        constexpr int PIECES = (NS / GI) * 64;
-        for (int id = threadIdx.x; id < PIECES; id += L::THREADS) {
-            const int rel = id >> 6, half = (id >> 5) & 1, row = id & 31;
-            const int slab = slab0 + rel;
-            uint4 v = make_uint4(0u, 0u, 0u, 0u);       // samples outside the row read as zero
-            if (slab >= 0 && slab < nslabs)
-                v = __ldg(reinterpret_cast<const uint4*>(in + ((int64_t)slab * a.na + k0 + row) * 32 + half * 16));
-            float2* dst = win + (rel * GI + half * (GI / 2)) * 32 + row;
-            if constexpr (TIn::ELEM_BYTES == 8) {
-                dst[0] = make_float2(__uint_as_float(v.x), __uint_as_float(v.y));
-                dst[32] = make_float2(__uint_as_float(v.z), __uint_as_float(v.w));
-            } else {
-                dst[0] = __half22float2(*reinterpret_cast<const __half2*>(&v.x));
-                dst[32] = __half22float2(*reinterpret_cast<const __half2*>(&v.y));
-                dst[64] = __half22float2(*reinterpret_cast<const __half2*>(&v.z));
-                dst[96] = __half22float2(*reinterpret_cast<const __half2*>(&v.w));
+        const char* src = in + ((int64_t)slab0 * a.na + k0 + lane) * 32;
+        const int64_t slab_bytes = (int64_t)a.na * 32;
+#pragma unroll
+        for (int id = 0; id < (NS / GI) * 2; id += L::THREADS / 32) {
+            const int piece = id + w;                    // (slab, half)
+            if ((NS / GI) * 2 % (L::THREADS / 32) == 0 || piece < (NS / GI) * 2) {
+                const int rel = piece >> 1, half = piece & 1;
+                uint4 v = make_uint4(0u, 0u, 0u, 0u);   // samples outside the row read as zero
+                if ((unsigned)(slab0 + rel) < (unsigned)nslabs)
+                    v = __ldg(reinterpret_cast<const uint4*>(src + rel * slab_bytes + half * 16));
+                put(win + (rel * GI + half * (GI / 2)) * PITCH + lane, v);
             }
         }
     }
@@ -471,25 +504,27 @@ __global__ void __launch_bounds__(RcmcSlab<TIn, TOut>::THREADS) sar_rcmc_filter_
             i0[p] += 1;
         }
     }
+    float2 wt[2][8];                                     // [pixel pair][tap], lanes x / y = the two pixels
+    sinc8_weights_pair(mu[0], mu[1], wt[0]);
+    sinc8_weights_pair(mu[2], mu[3], wt[1]);
     const float2* col = win + lane;
     float2 acc[4];
     auto taps = [&](int p, const float2* u) {            // u[0..7]: the eight samples of pixel p, tap j = -3 first
-        float wt[8];
-        sinc8_weights_rcp(mu[p], wt);
-        float2 s = make_float2(0.f, 0.f);
+        float2 sum = make_float2(0.f, 0.f);
 #pragma unroll
         for (int tap = 0; tap < 8; ++tap) {
-            const float ww = ((tap - 3) & 1) ? -wt[tap] : wt[tap];
-            s.x = fmaf(ww, u[tap].x, s.x);
-            s.y = fmaf(ww, u[tap].y, s.y);
+            const float m = (p & 1) ? wt[p >> 1][tap].y : wt[p >> 1][tap].x;
+            const float ww = ((tap - 3) & 1) ? -m : m;
+            sum.x = fmaf(ww, u[tap].x, sum.x);
+            sum.y = fmaf(ww, u[tap].y, sum.y);
         }
-        acc[p] = s;
+        acc[p] = sum;
     };
     if (i0[3] == i0[0]) {                                // the usual case: one window of 11 samples serves all four
         const int o = min(max(n + i0[0] - 3 - s0, 0), NS - 11);
         float2 u[11];
 #pragma unroll
-        for (int i = 0; i < 11; ++i) u[i] = col[(o + i) * 32];
+        for (int i = 0; i < 11; ++i) u[i] = col[(o + i) * PITCH];
 #pragma unroll
         for (int p = 0; p < 4; ++p) taps(p, u + p);
     } else {
@@ -498,7 +533,7 @@ __global__ void __launch_bounds__(RcmcSlab<TIn, TOut>::THREADS) sar_rcmc_filter_
             const int o = min(max(n + p + i0[p] - 3 - s0, 0), NS - 8);
             float2 u[8];
 #pragma unroll
-            for (int i = 0; i < 8; ++i) u[i] = col[(o + i) * 32];
+            for (int i = 0; i < 8; ++i) u[i] = col[(o + i) * PITCH];
             taps(p, u);
         }
     }
@@ -509,16 +544,18 @@ __global__ void __launch_bounds__(RcmcSlab<TIn, TOut>::THREADS) sar_rcmc_filter_
         acc[p] = cmul(acc[p], f);
         if (p < 3) f = cmul(f, step);                    // one more range bin: times exp(j 2 pi B)
     }
-    if constexpr (TOut::ELEM_BYTES == 8) {
-        float4* o = reinterpret_cast<float4*>(reinterpret_cast<float2*>(a.out) + slab_index(k, n, a.na, GO));
-        o[0] = make_float4(acc[0].x, acc[0].y, acc[1].x, acc[1].y);
-        o[1] = make_float4(acc[2].x, acc[2].y, acc[3].x, acc[3].y);
-    } else {
-        __half2 h[4];
+    {
+        if constexpr (TOut::ELEM_BYTES == 8) {
+            float4* o = reinterpret_cast<float4*>(reinterpret_cast<float2*>(a.out) + slab_index(k, n, a.na, GO));
+            o[0] = make_float4(acc[0].x, acc[0].y, acc[1].x, acc[1].y);
+            o[1] = make_float4(acc[2].x, acc[2].y, acc[3].x, acc[3].y);
+        } else {
+            __half2 h[4];
 #pragma unroll
-        for (int p = 0; p < 4; ++p) h[p] = __float22half2_rn(acc[p]);
-        *reinterpret_cast<uint4*>(reinterpret_cast<__half2*>(a.out) + slab_index(k, n, a.na, GO)) =
-            *reinterpret_cast<const uint4*>(h);
+            for (int p = 0; p < 4; ++p) h[p] = __float22half2_rn(acc[p]);
+            *reinterpret_cast<uint4*>(reinterpret_cast<__half2*>(a.out) + slab_index(k, n, a.na, GO)) =
+                *reinterpret_cast<const uint4*>(h);
+        }
     }
 }
 
@@ -595,11 +632,11 @@ cudaError_t launch_rcmc(const SarArgs& a, cudaStream_t st) {
     g_launch_count.fetch_add(1, std::memory_order_relaxed);
     return cudaGetLastError();
 }
-template <class T>
-cudaError_t launch_rcmc_slab(const SarArgs& a, cudaStream_t st) {
-    using L = RcmcSlab<T, T>;
+template <class TI, class TO>
+cudaError_t launch_rcmc_pass(const SarArgs& a, cudaStream_t st) {
+    using L = RcmcPass<TI, TO>;
     const unsigned grid = (unsigned)((a.na / L::ROWS) * (a.nr / L::NC));
-    sar_rcmc_filter_slab_kernel<T, T><<<grid, L::THREADS, 0, st>>>(a);
+    sar_rcmc_filter_slab_kernel<TI, TO><<<grid, L::THREADS, 0, st>>>(a);
     g_launch_count.fetch_add(1, std::memory_order_relaxed);
     return cudaGetLastError();
 }
@@ -630,8 +667,8 @@ static const SarEntry* find(const SarEntry (&tab)[K], int n, int dtype, bool sla
     return nullptr;
 }
 
-// largest spread of the integer shift inside one CTA of the slab row pass (32 Doppler bins x NC range
-// bins), over the whole image, in float64
+// largest spread of the integer shift inside one CTA of the row pass (32 Doppler bins x NC range bins),
+// over the whole image, in float64
 static double slab_shift_spread(const sar_rda_desc* d, int nc) {
     const double wavelength = kLight / d->carrier_hz, dr = kLight / (2.0 * d->fs_hz);
     const int na = (int)d->n_azimuth, nr = (int)d->n_range;
@@ -715,10 +752,19 @@ extern "C" int sar_rda_params_create(sar_rda_params_t* params, const sar_rda_des
     const int na = (int)d->n_azimuth, nr = (int)d->n_range, dt = d->intermediate_dtype;
     p->range = find(k_range, nr, dt, false);
     p->range_slab = find(k_range, nr, dt, true);
-    // Column tiles. With fp16 intermediates the wider tile on a cluster of two CTAs (32-byte instead of 16-byte
-    // row segments at n_azimuth = 4096: 84 -> 77 us); with complex64 the 4-column tile measured faster inside the
-    // chain (85 against 88 us per pass), where part of the image still sits in L2.
+    // Column tiles of the row-major layout: the persistent streaming kernel where it is compiled (4096 rows) and
+    // the image gives every multiprocessor several tiles; else, with fp16 intermediates, the wider tile on a
+    // cluster of two CTAs (32-byte instead of 16-byte row segments); else the plain 4-column tile.
+    int sms = 148;
+    {
+        int dev = 0;
+        if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    }
     auto cols_kernel = [&](bool inverse, int dtype) {
+        if (nr / 4 > sms) {
+            const KernelEntry* k = find_cols_kernel(na, inverse, dtype, dtype, 0, VAR_STREAM);
+            if (k && k->n >= 4096 && nr % k->w == 0) return k;
+        }
         if (dtype == B200FFT_C32H) {
             const KernelEntry* k = find_cols_kernel(na, inverse, dtype, dtype, 0, VAR_WIDE_CLUSTER);
             if (k && nr % k->w == 0) return k;
@@ -733,17 +779,18 @@ extern "C" int sar_rda_params_create(sar_rda_params_t* params, const sar_rda_des
         p->azfft_slab[i] = find_sar_cols_kernel(na, 2 << i, false, dt, dt);
         p->azifft_slab[i] = find_sar_cols_kernel(na, 2 << i, true, dt, B200FFT_C64);
     }
-    {   // the row pass stages COLS + HALO samples: the shift may grow by at most HALO - 16 bins over COLS bins
+    using RS = RcmcPass<StoreC64, StoreC64>;
+    // the slab row pass stages NC + HALO samples per row: the integer shift may spread by MAX_SPREAD inside a CTA
+    const bool row_pass_ok = na % 64 == 0 && nr % RS::NC == 0 && slab_shift_spread(d, RS::NC) + 2.0 <= (double)RS::MAX_SPREAD;
+    {   // the row-major row pass stages COLS + HALO samples: the shift may grow by at most HALO - 16 bins over COLS bins
         const double aa = wavelength * d->prf_hz / (4.0 * d->velocity_mps), u = aa * aa, sq = sqrt(1.0 - u);
         const double gmax = u / ((1.0 + sq) * sq);
         p->can_unfuse = p->azifft != nullptr && nr % RcmcRows::COLS == 0 &&
                         gmax * RcmcRows::COLS + 16.0 <= (double)RcmcRows::HALO;
     }
-    using RS = RcmcSlab<StoreC64, StoreC64>;
     p->can_slab = p->range_slab && p->rcmc_slab && p->azfft_slab[0] && p->azfft_slab[1] && p->azifft_slab[0] &&
-                  p->azifft_slab[1] && na % 64 == 0 && nr % RS::NC == 0 &&
-                  slab_shift_spread(d, RS::NC) + 2.0 <= (double)RS::MAX_SPREAD;
-    p->layout = p->can_slab ? 1 : 0;
+                  p->azifft_slab[1] && row_pass_ok;
+    p->layout = 0;
     p->tile_columns = 2;
     p->fused = p->layout == 0 && !p->can_unfuse;
     if (!p->range || !p->azfft || !p->rcmc || d->n_azimuth > 16384 || d->n_range > 16384 || nr % p->rcmc->w) {
@@ -853,7 +900,8 @@ extern "C" int sar_rda_run_step(const void* raw, sar_rda_params_t p, void* out, 
     f.prefetch_ahead = 0;
     if (slab) {
         a.out = buf1;
-        cudaError_t e = dt == B200FFT_C64 ? launch_rcmc_slab<StoreC64>(a, st) : launch_rcmc_slab<StoreC32H>(a, st);
+        cudaError_t e = dt == B200FFT_C64 ? launch_rcmc_pass<StoreC64, StoreC64>(a, st)
+                                          : launch_rcmc_pass<StoreC32H, StoreC32H>(a, st);
         if (e != cudaSuccess) return B200FFT_ERR_CUDA;
         const KernelEntry* k = p->azifft_slab[p->tile_columns == 4];
         f.in = buf1; f.out = out;

@@ -20,8 +20,8 @@ def _need_gpu():
 
 
 def _gpu_chain(scene, raw, dtype, steps=False, fused=None, layout=None, tile_columns=None):
-    """Run the chain through the C ABI. layout: 0 = row-major intermediates, 1 = slab layout (the
-    default); tile_columns: range bins per column tile on the slab layout."""
+    """Run the chain through the C ABI. layout: 0 = row-major intermediates (the default), 1 = slab layout (the
+     is 0); tile_columns: range bins per column tile on the slab layout."""
     import torch
     from paper_2609_32237_b200 import binding as B
     p = B.sar_rda_params_create(B.sar_desc_from_scene(scene, dtype))
@@ -41,7 +41,7 @@ def _gpu_chain(scene, raw, dtype, steps=False, fused=None, layout=None, tile_col
         rd = to_device_c64(raw)
         out = torch.zeros_like(rd)
         st = torch.cuda.current_stream().cuda_stream
-        slab = layout is None or layout == 1
+        slab = layout == 1
 
         def ws_as_complex():
             """The first intermediate image as a row-major complex128 matrix (undoing the slab
@@ -126,6 +126,36 @@ def test_small_scene_fused_and_unfused_step2_agree(small_scene, dtype, tol, layo
     for cell in sc.targets:
         assert quality.peak_cell(a, tuple(cell)) == tuple(cell)
         assert quality.peak_cell(b, tuple(cell)) == tuple(cell)
+
+
+def test_form_image_from_host_buffers(small_scene):
+    """sar_rda_form_image_host: raw data in pinned host memory, image back to pinned host memory,
+    copies and the chain ordered on one stream; same image as the device-resident call, bit for bit."""
+    import torch
+    from paper_2609_32237_b200 import binding as B
+    sc, raw, rc, S, img = small_scene
+    want = _gpu_chain(sc, raw, C64)
+    p = B.sar_rda_params_create(B.sar_desc_from_scene(sc, C64))
+    try:
+        need = B.sar_rda_workspace_bytes(p)
+        ws = torch.zeros(need, dtype=torch.uint8, device="cuda")
+        B.sar_rda_set_workspace(p, ws.data_ptr(), need)
+        h_raw = torch.from_numpy(np.ascontiguousarray(raw, dtype=np.complex64)).pin_memory()
+        h_out = torch.zeros_like(h_raw).pin_memory()
+        d_raw = torch.zeros(raw.shape, dtype=torch.complex64, device="cuda")
+        d_out = torch.zeros_like(d_raw)
+        st = torch.cuda.current_stream().cuda_stream
+        B.sar_rda_form_image_host(h_raw.data_ptr(), p, h_out.data_ptr(), d_raw.data_ptr(), d_out.data_ptr(), st)
+        torch.cuda.synchronize()
+        got = h_out.numpy()
+        assert rel_l2(got, img) <= 1e-5
+        assert np.array_equal(got.view(np.uint64), want.view(np.uint64))
+        assert np.array_equal(d_raw.cpu().numpy(), raw.astype(np.complex64))
+        with pytest.raises(B.B200FftError) as e:               # null host pointer
+            B.sar_rda_form_image_host(0, p, h_out.data_ptr(), d_raw.data_ptr(), d_out.data_ptr(), st)
+        assert e.value.status == 1
+    finally:
+        B.sar_rda_params_destroy(p)
 
 
 def test_single_on_grid_echo_compresses_to_the_pulse_length():
