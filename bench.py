@@ -614,7 +614,8 @@ def run_others(torch, B, args, peak):
     h_img = torch.empty_like(h_raw).pin_memory()
     rd = h_raw.cuda()
     img = torch.empty_like(rd)
-    variants = {"": {}, "_slab_layout": {"layout": 1, "tile_columns": 4}, "_fused_step2": {"fused_rcmc": 1}}
+    variants = {"": {}, "_slab_layout": {"layout": 1, "tile_columns": 4}, "_fused_step2": {"fused_rcmc": 1},
+                "_via_transpose": {"layout": 2}}
     for dtype, base in ((0, "sar_4096x4096_fp32_intermediates"), (1, "sar_4096x4096_fp16_intermediates")):
         for suffix, opts in variants.items():
             p = B.sar_rda_params_create(B.sar_desc_from_scene(sc, dtype))

@@ -18,8 +18,14 @@ namespace b200fft {
 // plain loads. After the last stage the results go back to shared memory as a dense image (the exchange
 // buffer is free by then) and leave as TMA stores, which the next tile's first stage overlaps; the stores
 // must have read shared memory before the next exchange overwrites it (wait_group.read). Tensor maps cover
-// this GPU's own memory; no multicast. (Two-column tiles at two CTAs per multiprocessor, i.e. boxes with
-// 16-byte rows, measured twice as slow: 144 against 74 us on 4096 x 4096.) Every wait is bounded: a CTA whose wait runs out raises
+// this GPU's own memory; no multicast. Measured on 4096 x 4096 complex64: 74 us against 92 us for the plain
+// kernel. Variants that were built, tested and measured without gain, and dropped: two-column tiles at two CTAs
+// per multiprocessor, i.e. boxes with 16-byte rows (144 us); two warp groups of two columns each that take
+// turns on one 64 KiB exchange buffer, so that one group computes while the other exchanges, with the whole
+// next tile staged (76 us, the same with the 32-byte swizzle against the bank conflicts of its half-row
+// accesses, and 74 us on contiguous tiles moved as 64 KiB boxes: the time is set by the traffic through shared
+// memory, about 1 MiB per 128 KiB tile with the staging on both ends, not by the access pattern in main
+// memory). Every wait is bounded: a CTA whose wait runs out raises
 // g_tma_timeouts once, stops taking tiles, waits (bounded again) for the copies it still has in flight
 // and returns; the output of that call is then incomplete.
 __device__ int g_tma_timeouts = 0;   // CTAs whose wait for a copy ran out of polls (never expected)
@@ -166,8 +172,7 @@ static EncodeTiledFn encode_tiled_fn() {
     }
     return fn;
 }
-// a rows x ld matrix of elem_bytes-sized complex elements seen as 4-byte words, boxes of box_rows rows x w elements
-static bool make_column_map(CUtensorMap* m, const void* base, int64_t rows, int64_t ld, int w, int box_rows, int elem_bytes) {
+bool make_column_map(CUtensorMap* m, const void* base, int64_t rows, int64_t ld, int w, int box_rows, int elem_bytes) {
     EncodeTiledFn fn = encode_tiled_fn();
     if (!fn) return false;
     const int words = elem_bytes / 4;

@@ -1,5 +1,6 @@
 // Host-side table of compiled kernel variants.
 #pragma once
+#include <cuda.h>
 #include <cuda_runtime.h>
 #include <atomic>
 #include <cstdint>
@@ -115,6 +116,9 @@ EntryList rows_entries_small();     // N = 32 .. 2048
 EntryList rows_entries_large();     // N = 4096 .. 16384 and the alternative factorisations
 EntryList rows_entries_cluster();   // transforms shared by a cluster of CTAs
 EntryList cols_entries_more();      // column tiles on clusters, wide column tiles
+// a rows x ld matrix of elem_bytes-sized complex elements as a 2-D tensor map of 4-byte words, boxes of
+// box_rows rows x w elements (cuTensorMapEncodeTiled through the runtime's driver entry point)
+bool make_column_map(CUtensorMap* m, const void* base, int64_t rows, int64_t ld, int w, int box_rows, int elem_bytes);
 
 // cl: CTAs per tile (cluster size); 0 picks the default for that size and batch (plain kernels only)
 const KernelEntry* find_rows_kernel(int n, bool inverse, int in_dtype, int out_dtype, int cl = 0,

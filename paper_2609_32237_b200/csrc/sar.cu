@@ -706,7 +706,12 @@ struct b200fft_sar_s {
     const KernelEntry* azfft_slab[2];    // forward column tiles of 2 and of 4 range bins, intermediate type both ways
     const KernelEntry* azifft_slab[2];   // inverse column tiles, intermediate type in, complex64 out
     bool can_slab;
-    int layout;                  // 0 row-major, 1 slab
+    // azimuth transforms by transposition ("layout" 2): the paper's four-pass form, as a measured comparison
+    const KernelEntry* rows_fwd;         // n_azimuth-point row transforms of the transposed image, intermediate type
+    const KernelEntry* rows_inv;         // the same, inverse, complex64
+    float2* tw_rows;
+    bool can_transpose;
+    int layout;                  // 0 row-major (direct column kernels), 1 slab, 2 row-major with transposes
     int tile_columns;            // slab layout: range bins per column tile, 2 or 4
     bool fused;                  // step 2 as one kernel (true) or as row pass + column pass (false)
     float2 *tw_range, *tw_az, *H;
@@ -719,6 +724,7 @@ struct b200fft_sar_s {
 static void sar_release(b200fft_sar_s* p) {
     if (p->tw_range) cudaFree(p->tw_range);
     if (p->tw_az) cudaFree(p->tw_az);
+    if (p->tw_rows) cudaFree(p->tw_rows);
     if (p->H) cudaFree(p->H);
     if (p->mig) cudaFree(p->mig);
     if (p->phs) cudaFree(p->phs);
@@ -790,8 +796,11 @@ extern "C" int sar_rda_params_create(sar_rda_params_t* params, const sar_rda_des
     }
     p->can_slab = p->range_slab && p->rcmc_slab && p->azfft_slab[0] && p->azfft_slab[1] && p->azifft_slab[0] &&
                   p->azifft_slab[1] && row_pass_ok;
+    p->rows_fwd = find_rows_kernel(na, false, dt, dt, 1, nr);
+    p->rows_inv = find_rows_kernel(na, true, B200FFT_C64, B200FFT_C64, 1, nr);
+    p->can_transpose = p->rows_fwd && p->rows_inv && p->rows_fwd->tw_total == p->rows_inv->tw_total && p->can_unfuse;
     p->layout = 0;
-    p->tile_columns = 2;
+    p->tile_columns = 4;
     p->fused = p->layout == 0 && !p->can_unfuse;
     if (!p->range || !p->azfft || !p->rcmc || d->n_azimuth > 16384 || d->n_range > 16384 || nr % p->rcmc->w) {
         delete p;
@@ -821,6 +830,9 @@ extern "C" int sar_rda_params_create(sar_rda_params_t* params, const sar_rda_des
     const double dr = kLight / (2.0 * d->fs_hz);
     const double kappa = (d->bandwidth_hz / d->pulse_s) / (d->fs_hz * d->fs_hz);
     ok = p->range->build_tw(p->tw_range, 0) == cudaSuccess && p->rcmc->build_tw(p->tw_az, 0) == cudaSuccess;
+    if (ok && p->can_transpose)
+        ok = cudaMalloc(&p->tw_rows, sizeof(float2) * (size_t)p->rows_fwd->tw_total) == cudaSuccess &&
+             p->rows_fwd->build_tw(p->tw_rows, 0) == cudaSuccess;
     sar_build_matched_filter<<<(nr + 127) / 128, 128>>>(p->H, nr, (int)pulse_samples, kappa);
     sar_build_doppler_tables<<<(na + 127) / 128, 128>>>(p->mig, p->phs, p->stp, na, nr, wavelength, d->prf_hz,
                                                        d->velocity_mps, d->r_center_m, dr);
@@ -877,6 +889,42 @@ extern "C" int sar_rda_run_step(const void* raw, sar_rda_params_t p, void* out, 
         a.tiles = na; a.ld = nr; a.nr = (int)nr; a.na = (int)na; a.scale = 1.0f;
         return ok((slab ? p->range_slab : p->range)->launch(a, st));
     }
+    if (p->layout == 2 && step >= 1) {
+        // The paper's four-pass form: an azimuth transform is a transpose, transforms along the (now contiguous)
+        // rows, and a transpose back. Step 1 goes workspace -> second half -> workspace; step 2 runs the row pass
+        // into `out`, then takes the whole workspace as one complex64 image for the inverse transform.
+        const int eb = dt == B200FFT_C64 ? 8 : 4;
+        FftArgs f{};
+        f.tw = p->tw_rows;
+        f.tiles = nr; f.dist = na;
+        f.prefetch_ahead = 0;
+        if (step == 1) {
+            if (transpose_launch(buf0, buf1, (int)na, (int)nr, nr, na, eb, st) != cudaSuccess) return B200FFT_ERR_CUDA;
+            f.in = buf1; f.out = buf1;
+            f.scale = (float)(1.0 / (double)na);
+            if (p->rows_fwd->launch(f, st) != cudaSuccess) return B200FFT_ERR_CUDA;
+            return ok(transpose_launch(buf1, buf0, (int)nr, (int)na, na, nr, eb, st));
+        }
+        if (!out) return B200FFT_ERR_INVALID_ARG;
+        if (reinterpret_cast<uintptr_t>(out) % 16) return B200FFT_ERR_ALIGNMENT;
+        SarArgs a{};
+        a.in = buf0; a.out = out; a.tw = p->tw_az;
+        a.tab = SarTables{p->H, p->mig, p->phs, p->stp};
+        a.ld = nr; a.nr = (int)nr; a.na = (int)na; a.scale = 1.0f;
+        const int chunks = (int)(nr / RcmcRows::COLS);
+        if (dt == B200FFT_C64)
+            sar_rcmc_filter_rows_kernel<StoreC64><<<(unsigned)(na * chunks), RcmcRows::TPB, 0, st>>>(a, chunks);
+        else
+            sar_rcmc_filter_rows_kernel<StoreC32H><<<(unsigned)(na * chunks), RcmcRows::TPB, 0, st>>>(a, chunks);
+        g_launch_count.fetch_add(1, std::memory_order_relaxed);
+        if (cudaGetLastError() != cudaSuccess) return B200FFT_ERR_CUDA;
+        if (2 * image_bytes(p) < (size_t)na * (size_t)nr * 8) return B200FFT_ERR_WORKSPACE;
+        if (transpose_launch(out, buf0, (int)na, (int)nr, nr, na, 8, st) != cudaSuccess) return B200FFT_ERR_CUDA;
+        f.in = buf0; f.out = buf0;
+        f.scale = 1.0f;                     // 1/n_azimuth was applied after the forward azimuth FFT
+        if (p->rows_inv->launch(f, st) != cudaSuccess) return B200FFT_ERR_CUDA;
+        return ok(transpose_launch(buf0, out, (int)nr, (int)na, na, nr, 8, st));
+    }
     if (step == 1) {
         FftArgs a{};
         a.in = buf0; a.out = buf0; a.tw = p->tw_az;
@@ -926,14 +974,16 @@ extern "C" int sar_rda_set_option(sar_rda_params_t p, const char* key, int64_t v
     if (!p || !key) return B200FFT_ERR_INVALID_ARG;
     if (std::strcmp(key, "fused_rcmc") == 0) {
         if (!value && p->layout == 0 && !p->can_unfuse) return B200FFT_ERR_UNSUPPORTED;
+        if (value && p->layout == 2) return B200FFT_ERR_UNSUPPORTED;
         p->fused = value != 0;
         return B200FFT_OK;
     }
     if (std::strcmp(key, "layout") == 0) {
-        if (value != 0 && value != 1) return B200FFT_ERR_INVALID_ARG;
-        if (value == 1 && !p->can_slab) return B200FFT_ERR_UNSUPPORTED;
+        if (value < 0 || value > 2) return B200FFT_ERR_INVALID_ARG;
+        if ((value == 1 && !p->can_slab) || (value == 2 && !p->can_transpose)) return B200FFT_ERR_UNSUPPORTED;
         p->layout = (int)value;
         if (value == 0 && !p->can_unfuse) p->fused = true;
+        if (value == 2) p->fused = false;
         return B200FFT_OK;
     }
     if (std::strcmp(key, "tile_columns") == 0) {

@@ -298,7 +298,7 @@ def test_table_twiddles_variant_matches():
 
 @pytest.mark.parametrize("n,cols,ld,dtype", [(2048, 16, 24, C64), (4096, 16, 24, C64), (4096, 1236, 1240, C64),
                                              (4096, 16, 24, C32H), (4096, 1236, 1240, C32H)])
-def test_columns_streaming_kernel(n, cols, ld, dtype):
+def test_columns_streaming_kernel(n, cols, ld, dtype, kind=1):
     """The persistent column kernel whose tiles arrive and leave through the tensor memory
     accelerator (plan option "stream"; the default for large 4096-row matrices): sampled columns
     against the oracle, everything against the plain-load kernel, padding untouched, in place,
@@ -317,7 +317,7 @@ def test_columns_streaming_kernel(n, cols, ld, dtype):
             dev = to_device_half(h)
             src = inputs.from_half_storage(h)
         want = oracle.fft_cols(src[:, pick], direction)
-        got_t = run_fft(dev, n, cols, ld, 1, direction, dtype, options={"stream": 1})
+        got_t = run_fft(dev, n, cols, ld, 1, direction, dtype, options={"stream": kind})
         plain_t = run_fft(dev, n, cols, ld, 1, direction, dtype, options={"stream": 0, "cluster": 1})
         if dtype == C64:
             got, plain = got_t.cpu().numpy(), plain_t.cpu().numpy()
@@ -327,12 +327,12 @@ def test_columns_streaming_kernel(n, cols, ld, dtype):
         assert per_col.max() <= tol
         assert rel_l2(got[:, :cols], plain[:, :cols]) <= (2e-7 if dtype == C64 else 2e-4)
         assert np.all(got[:, cols:] == 0)
-        inplace = run_fft(dev.clone(), n, cols, ld, 1, direction, dtype, inplace=True, options={"stream": 1})
+        inplace = run_fft(dev.clone(), n, cols, ld, 1, direction, dtype, inplace=True, options={"stream": kind})
         assert bool((inplace[:, :cols] == got_t[:, :cols]).all())
     assert B.tma_timeouts() == _timeouts_at_start(B)
 
 
-def test_bounded_wait_gives_up_and_the_gpu_stays_usable():
+def test_bounded_wait_gives_up_and_the_gpu_stays_usable(kind=1):
     """The streaming kernel's wait for its copies is bounded. With the test knob "starve_wait" the
     consumer polls a barrier that nothing ever completes (the copies themselves are counted on
     another one and do land), and with "wait_polls" the limit is 1024 polls: every CTA gives up
@@ -343,12 +343,12 @@ def test_bounded_wait_gives_up_and_the_gpu_stays_usable():
     n, cols = 4096, 24                       # six tiles, six CTAs
     m = inputs.uniform_complex64((n, cols), 37)
     before = B.tma_timeouts()
-    out = run_fft(to_device_c64(m), n, cols, cols, 1, FWD, C64, options={"stream": 1, "starve_wait": 1, "wait_polls": 1024})
+    out = run_fft(to_device_c64(m), n, cols, cols, 1, FWD, C64, options={"stream": kind, "starve_wait": 1, "wait_polls": 1024})
     torch.cuda.synchronize()
     assert B.tma_timeouts() - before == 6
     assert bool((out == 0).all())            # nothing was transformed, nothing written
     want = oracle.fft_cols(m.astype(np.complex128), FWD)
-    got = run_fft(to_device_c64(m), n, cols, cols, 1, FWD, C64, options={"stream": 1}).cpu().numpy()
+    got = run_fft(to_device_c64(m), n, cols, cols, 1, FWD, C64, options={"stream": kind}).cpu().numpy()
     assert np.max(np.linalg.norm(got - want, axis=0) / np.linalg.norm(want, axis=0)) <= TOL32
     assert B.tma_timeouts() - before == 6    # the ordinary call raised nothing
 
