@@ -100,40 +100,47 @@ int fft_execute_host(fft_plan_t plan, const void *host_in, void *host_out,
 /* Free the plan's tables. The caller must have synchronised outstanding work. */
 int fft_plan_destroy(fft_plan_t plan);
 
-/* Test knob: force a kernel variant (paper, Section "One Pass": "a regression
- * test forces N=8192 through this path"). key "four_step" value 1 routes a
- * rows plan of any supported n >= 4096 through the two-pass split (value 0
- * brings a plan of n <= 32768 back to its single pass). Key
- * "cluster" value c (1, 2 or 4; 0 = the default for that size) picks the
- * variant of a single-pass plan in which c CTAs of one thread-block cluster
- * share a tile through distributed shared memory; B200FFT_ERR_UNSUPPORTED if
- * that variant is not compiled for the plan's size. (Defaults: rows of
- * n = 16384 / 8192 with at most 32 / 16 transforms, and rows of n = 32768, are
- * split over clusters; columns plans take the widest tile whose width divides
- * the batch: 16 columns for n <= 512, 8 for n = 1024, and for n >= 2048 a tile
- * of 32768 / n columns shared by a cluster of two CTAs, except complex64 at
- * n = 2048; value 1 forces the single-CTA 4-column tile, 2 columns at 8192.)
- * Key "prefetch" value d
- * makes each CTA of a rows plan ask L2 for the input of the transform d tiles
- * ahead (0 = off, -1 = the default: one wave ahead for n = 16384). Key "tma"
- * value 1 makes a complex64 columns plan (n = 1024, 2048, 4096) stage its tiles
- * through the tensor memory accelerator (2-D tiled bulk copies, no multicast)
- * instead of plain vector loads and stores; same results. Key "staged" value
- * 1 makes a rows plan with n = 16384 run as a persistent kernel (one CTA per
- * multiprocessor looping over transforms) whose next transform arrives in
- * shared memory through untiled bulk copies while the current one is computed;
- * 0 forbids it, -1 restores the default (on for fp16 storage with a batch of
- * at least two transforms per multiprocessor); B200FFT_ERR_UNSUPPORTED for
- * other sizes; same results. Every wait on such a copy is bounded:
- * b200fft_tma_timeouts() counts waits that gave up. Key "via_transpose" value
- * 1 makes a columns plan work the way the paper's four-pass pipeline does
- * (Section "End to End": a transpose, then the transform along rows) instead
- * of reading the columns directly: transpose into the workspace, row
- * transforms in place there, transpose back into `out`; it then needs a
- * workspace of n*batch elements of the storage type (set_workspace), which
- * must be neither `in` nor `out`; same results; kept as a measured comparison
- * with the direct column kernel. Unknown keys return
- * B200FFT_ERR_INVALID_ARG. Must be called before set_workspace. */
+/* Variant choice and test knobs (paper, Section "One Pass": "a regression test forces N=8192 through
+ * this path"). Every variant of a plan gives the same results to rounding. Unknown keys return
+ * B200FFT_ERR_INVALID_ARG; a variant that is not compiled for the plan's size returns
+ * B200FFT_ERR_UNSUPPORTED and leaves the plan as it was. Call before set_workspace.
+ *   "four_step"  1 routes a rows plan of any supported n >= 4096 through the two-pass split; 0 brings a
+ *                plan of n <= 32768 back to its single pass.
+ *   "cluster"    c = 1, 2 or 4 (0 = the default rules; other values are B200FFT_ERR_INVALID_ARG): the
+ *                single-pass variant in which c CTAs of one thread-block cluster share a tile through
+ *                distributed shared memory. Defaults: rows of n = 16384 / 8192 with at most 32 / 16
+ *                transforms, and rows of n = 32768, are split over clusters. Columns plans take, in
+ *                this order, the widest tile that is compiled and divides the batch: 16 columns for
+ *                n <= 512 and 8 for n = 1024; the streaming kernel (see "stream") for n = 4096 when the
+ *                matrix has more than one 4-column tile per multiprocessor; for other n >= 2048 a
+ *                tile of 32768 / n columns shared by a cluster of two CTAs (not complex64 at n = 2048);
+ *                "cluster" = 1 forces the plain single-CTA 4-column tile (2 columns at n = 8192).
+ *   "stream"     (columns plans; "tma" is an alias) 1 selects the persistent streaming kernel (n = 2048
+ *                complex64, n = 4096 both storage types): one CTA per multiprocessor loops over
+ *                4-column tiles, and the tensor memory accelerator brings the next tile into shared
+ *                memory (2-D tiled bulk copies of this GPU's own memory, no multicast) and takes the
+ *                finished one out while the current one is transformed; 0 forbids it; -1 restores the
+ *                default rules.
+ *   "staged"     (rows plans, n = 16384) 1 selects the persistent kernel whose next transform arrives
+ *                in shared memory through untiled bulk copies while the current one is computed; 0
+ *                forbids it; -1 restores the default (on for fp16 storage with at least two transforms
+ *                per multiprocessor).
+ *   "prefetch"   d makes each CTA of a rows plan ask L2 for the input of the transform d tiles ahead
+ *                (0 = off, -1 = the default: one wave ahead for n = 16384).
+ *   "via_transpose"  1 makes a columns plan work the way the paper's four-pass pipeline does (Section
+ *                "End to End": a transpose, then the transform along rows): transpose into the
+ *                workspace, row transforms in place there, transpose back into `out`; it then needs a
+ *                workspace of n*batch elements of the storage type, which must be neither `in` nor
+ *                `out`; kept as a measured comparison with the direct column kernels.
+ *   "alt_factorisation"  (rows plans, test knob) 1 selects the other compiled factorisation: n = 4096
+ *                with every first-stage twiddle row loaded from its table instead of multiplied up,
+ *                n = 16384 as 16 x 4 x 16 x 16 instead of 32 x 32 x 16.
+ *   "wait_polls", "starve_wait"  (test knobs of the kernels that wait on asynchronous copies) every such
+ *                wait is bounded: after wait_polls polls (0 = the default, 2^22, a fraction of a second)
+ *                the CTA gives up, raises the counter that b200fft_tma_timeouts() reads, waits for the
+ *                copies it still has in flight and returns; the output of that call is then incomplete.
+ *                starve_wait = 1 makes the streaming kernel poll a barrier that nothing completes, so
+ *                that a test can see the give-up path run; never set it otherwise. */
 int fft_plan_set_option(fft_plan_t plan, const char *key, int64_t value);
 
 /* The paper has no counterpart to this call. It is for callers that must not
@@ -184,10 +191,11 @@ const char *fft_status_string(int status);
  * (all plans, all streams); for launch accounting in benchmarks. */
 int64_t b200fft_launch_count(void);
 
-/* Number of mbarrier waits in the TMA column variant and the staged rows
- * variant that gave up after their poll limit since the library was loaded (synchronises the device; 0 unless
- * something is badly wrong: the waits are bounded so that a lost copy can never
- * hang the GPU). */
+/* Number of bounded waits on asynchronous copies (streaming column kernel:
+ * counted once per CTA; staged rows kernel) that gave up after their poll limit
+ * since the library was loaded. Synchronises the device. 0 unless something is
+ * badly wrong or a test asked for it: the waits are bounded so that a lost copy
+ * can never hang the GPU. */
 int b200fft_tma_timeouts(void);
 
 /* ------------------------------------------------------------------------
@@ -196,14 +204,18 @@ int b200fft_tma_timeouts(void);
  * chirp spectrum, inverse FFT along each pulse, 1/n_range included); azimuth
  * FFT along each range bin; range cell migration correction with an 8-tap
  * sinc interpolator; the azimuth filter exp(+j 4 pi R0 (D - 1) / lambda),
- * D = sqrt(1 - (lambda f_a / 2 v)^2); azimuth inverse FFT. Three passes over
- * memory: fused range compression; column FFT; fused RCMC + filter + inverse
- * column FFT (or, by default where the scene allows, RCMC + filter along the
- * rows followed by the inverse column FFT in place: see sar_rda_set_option).
+ * D = sqrt(1 - (lambda f_a / 2 v)^2); azimuth inverse FFT. The chirp is an
+ * up-chirp with its replica centred on t = 0, and range bin n_range/2 is the
+ * scene centre (both fixed; the descriptor has no field for them). The default
+ * form is four kernels: fused range compression; the azimuth FFT read as
+ * columns in place (scaled 1/n_azimuth); RCMC + filter along the rows, written
+ * to `out`; the inverse azimuth FFT as columns of `out` in place. The paper's
+ * three-pass form (RCMC + filter + inverse FFT fused on column tiles) and two
+ * other organisations are selectable: see sar_rda_set_option.
  * ---------------------------------------------------------------------- */
 typedef struct {
-    int64_t n_azimuth;          /* pulses (rows); power of two, 256..16384 */
-    int64_t n_range;            /* range samples per pulse (columns); power of two, 256..16384 */
+    int64_t n_azimuth;          /* pulses (rows): 1024, 2048 or 4096 */
+    int64_t n_range;            /* range samples per pulse (columns): 1024, 2048, 4096 or 8192 */
     double carrier_hz;
     double bandwidth_hz;        /* chirp bandwidth; up-chirp, replica centred on t = 0 */
     double fs_hz;               /* range sampling rate */
@@ -220,24 +232,36 @@ typedef struct {
  * Synchronises the device once. */
 int sar_rda_params_create(sar_rda_params_t *params, const sar_rda_desc *desc);
 
-/* Bytes of DEVICE workspace: one intermediate image of n_azimuth*n_range
- * elements of the intermediate dtype (the azimuth FFT runs in place on it). */
+/* Bytes of DEVICE workspace: two intermediate images of n_azimuth*n_range
+ * elements of the intermediate dtype (the default chain uses the first; the
+ * slab and transposed forms use both). Its contents between calls are
+ * unspecified; its layout is the library's own. */
 int sar_rda_workspace_bytes(sar_rda_params_t params, size_t *bytes);
 int sar_rda_set_workspace(sar_rda_params_t params, void *device_ptr, size_t bytes);
 
-/* Variant choice. Key "fused_rcmc": 1 runs step 2 as the single fused kernel
- * (RCMC + filter + inverse azimuth FFT on column tiles: three passes over
- * memory in all); 0 runs it as a row pass (RCMC + filter, written to `out`)
- * followed by the in-place inverse column FFT of `out` (four passes, but
- * faster on B200; the default whenever the scene allows it). Both give the
- * same image to rounding. B200FFT_ERR_UNSUPPORTED if the unfused form cannot
- * serve this scene (migration growing by more than 48 bins over 1024 range
- * bins, or n_range not a multiple of 1024). */
+/* Variant choice; every form gives the same image to rounding.
+ *   "fused_rcmc"   1 runs step 2 as the single fused kernel (RCMC + filter + inverse azimuth FFT on
+ *                  column tiles: three passes over memory in all, the paper's best form); 0 runs it as a
+ *                  row pass followed by the inverse column FFT (four passes, but faster on B200; the
+ *                  default whenever the scene allows it: B200FFT_ERR_UNSUPPORTED if the migration grows
+ *                  by more than 48 bins over 1024 range bins or n_range is not a multiple of 1024).
+ *   "layout"       0 (default) keeps the intermediate image row-major and transforms its columns
+ *                  directly. 1 keeps it in slabs of 32-byte granules (4 complex64 or 8 complex-half range
+ *                  bins; element (k, n) at ((n / G) * n_azimuth + k) * G + n % G), so that every column
+ *                  tile is row segments inside one contiguous slab; step 2 then goes slab to slab (second
+ *                  half of the workspace; with fp16 intermediates this image is fp16 as well, one more
+ *                  rounding) and the inverse column FFT writes the row-major image. 2 is the paper's
+ *                  four-pass form as a measured comparison: every azimuth transform is a transpose,
+ *                  transforms along rows, and a transpose back. B200FFT_ERR_UNSUPPORTED if the scene's
+ *                  shift spreads by more than 16 bins inside a block of 32 Doppler bins by 64 range bins
+ *                  (layout 1) or the row pass cannot serve it (layout 2).
+ *   "tile_columns" 2 or 4 (default): range bins per column tile on the slab layout. */
 int sar_rda_set_option(sar_rda_params_t params, const char *key, int64_t value);
 
 /* raw: DEVICE, n_azimuth x n_range interleaved complex fp32, row-major (row =
  * pulse). out: DEVICE, same shape and type, the focused image; must not alias
- * raw or the workspace. Enqueues three kernels on `stream`; does not
+ * raw or the workspace. Enqueues four kernels on `stream` (three with
+ * "fused_rcmc", eight with "layout" 2); does not
  * synchronise. Calls sharing one params object must not overlap on the GPU
  * (they share its workspace). */
 int sar_rda_form_image(const void *raw, sar_rda_params_t params, void *out, void *stream);
@@ -247,9 +271,10 @@ int sar_rda_form_image(const void *raw, sar_rda_params_t params, void *out, void
 int sar_rda_form_image_host(const void *host_raw, sar_rda_params_t params, void *host_out,
                             void *dev_raw, void *dev_out, void *stream);
 
-/* Run one step only, for tests: step 0 range compression (raw -> workspace),
- * 1 azimuth FFT (workspace, in place), 2 RCMC + filter + inverse FFT
- * (workspace -> out; one or two kernels, see sar_rda_set_option). `raw` is read by step 0 only, `out` written by step 2 only. */
+/* Run one step only, for tests: step 0 range compression (raw -> first image
+ * of the workspace), 1 azimuth FFT (that image, in place), 2 RCMC + filter +
+ * inverse FFT (-> out; one or more kernels, see sar_rda_set_option). `raw` is
+ * read by step 0 only, `out` written by step 2 only. */
 int sar_rda_run_step(const void *raw, sar_rda_params_t params, void *out, int step, void *stream);
 
 int sar_rda_params_destroy(sar_rda_params_t params);

@@ -49,6 +49,23 @@ __global__ void __launch_bounds__(C::THREADS, CPS)
     extern __shared__ __align__(128) float2 smem_stream[];   // TMA destinations and sources are 128-byte aligned
     constexpr int W = C::W, N = C::N, S = C::S;
     constexpr int XW_IN = W * TIn::ELEM_BYTES / 4, XW_OUT = W * TOut::ELEM_BYTES / 4;   // tile width in 4-byte map elements
+    using G1 = Geo<C, 1>;
+    using GS = Geo<C, S>;
+    constexpr int V = G1::V, r = G1::r, rs = GS::r, KS = N / rs;
+    static_assert(V == 2 && GS::V == 2 && (rs == 8 || rs == 16 || rs == 32), "one register pair per slot at both ends");
+    // When the staging buffer cannot hold the whole tile, the rows left to plain loads are the first-stage
+    // slots j = 3 mod 4: the composite butterfly consumes its inputs subset by subset (j = a + 4 b, a = 0..3),
+    // so these are needed last and their latency hides behind the arithmetic on the other three subsets.
+    constexpr bool ALL_STAGED = L::SBOX == L::NBOX;
+    constexpr bool SPLIT4 = !ALL_STAGED && G1::Ls == L::BOX_ROWS && r == 16 && L::SBOX >= 12;
+    static_assert(ALL_STAGED || SPLIT4, "a partly staged tile keeps three of every four first-stage slots");
+    constexpr int STAGED_BOXES = ALL_STAGED ? L::NBOX : 12;
+    // With fp16 storage the results leave in four batches (output rows k * KS + b0 with k = c mod 4, as soon as
+    // the last stage has emitted them), so that the copy engine reads the image while the rest is still being
+    // computed, and the first stage's arithmetic runs before the wait for the previous tile's stores (measured
+    // 62 -> 60 us on 4096 x 4096; with complex64 the same order measured slower, 74 -> 77 us, and is not used).
+    constexpr bool PROGRESSIVE = KS == L::BOX_ROWS && rs == 16 && TOut::ELEM_BYTES == 4;
+    constexpr int STORE_THREADS = PROGRESSIVE ? 4 : L::NBOX;
     __shared__ __align__(8) uint64_t bar[2];                  // [0] counts the copies; [1] is never completed
     const int t = threadIdx.x;
     float2* X = smem_stream;
@@ -56,10 +73,18 @@ __global__ void __launch_bounds__(C::THREADS, CPS)
     const int polls = a.wait_polls > 0 ? a.wait_polls : kDefaultWaitPolls;
 
     auto issue = [&](int64_t tile) {                          // thread 0: boxes of `tile` into the staging buffer
-        mbar_expect_tx(&bar[0], (unsigned)(L::SBOX * L::BOX_BYTES));
-        for (int b = 0; b < L::SBOX; ++b)
-            tma_load_2d(Sb + b * L::BOX_BYTES, &tm_in, (int)(tile * XW_IN), b * L::BOX_ROWS, &bar[0]);
-        for (int b = L::SBOX; b < L::NBOX; ++b) tma_prefetch_2d(&tm_in, (int)(tile * XW_IN), b * L::BOX_ROWS);
+        mbar_expect_tx(&bar[0], (unsigned)(STAGED_BOXES * L::BOX_BYTES));
+        if constexpr (ALL_STAGED) {
+            for (int b = 0; b < L::NBOX; ++b)
+                tma_load_2d(Sb + b * L::BOX_BYTES, &tm_in, (int)(tile * XW_IN), b * L::BOX_ROWS, &bar[0]);
+        } else {
+            for (int b = 0; b < L::NBOX; ++b) {
+                if ((b & 3) != 3)
+                    tma_load_2d(Sb + (b - (b >> 2)) * L::BOX_BYTES, &tm_in, (int)(tile * XW_IN), b * L::BOX_ROWS, &bar[0]);
+                else
+                    tma_prefetch_2d(&tm_in, (int)(tile * XW_IN), b * L::BOX_ROWS);
+            }
+        }
     };
     if (t == 0) {
         mbar_init(&bar[0], 1);
@@ -79,9 +104,6 @@ __global__ void __launch_bounds__(C::THREADS, CPS)
     for (; tile < a.tiles; tile += gridDim.x) {
         const int64_t next = tile + gridDim.x;
         asm volatile("" : "+r"(e.t));                         // keep the thread index opaque per tile (register pressure)
-        using G1 = Geo<C, 1>;
-        constexpr int V = G1::V, r = G1::r;
-        static_assert(V == 2, "one register pair per first-stage slot");
         const int c = C::template cidx<V>(e.t, 0, 0);
         const int q = c % W, lo = c / W;
         const int64_t gbase = tile * W;
@@ -94,7 +116,7 @@ __global__ void __launch_bounds__(C::THREADS, CPS)
         // rows that did not fit the staging buffer: plain loads (L2 was asked for them a tile ago)
         static_for<0, r>([&](auto j_) {
             constexpr int j = decltype(j_)::value;
-            if constexpr ((j * G1::Ls) / L::BOX_ROWS >= L::SBOX) {
+            if constexpr (!ALL_STAGED && (j & 3) == 3) {
                 TIn::load2(a.in, gbase + (int64_t)(j * G1::Ls + lo) * a.dist + q, e.x[j * V], e.x[j * V + 1]);
                 fix(j);
             }
@@ -105,24 +127,46 @@ __global__ void __launch_bounds__(C::THREADS, CPS)
         if (t == 0) in_flight = 0;
         static_for<0, r>([&](auto j_) {
             constexpr int j = decltype(j_)::value;
-            if constexpr ((j * G1::Ls) / L::BOX_ROWS < L::SBOX) {
+            if constexpr (ALL_STAGED) {
                 TIn::load2(Sb, (j * G1::Ls + lo) * W + q, e.x[j * V], e.x[j * V + 1]);
+                fix(j);
+            } else if constexpr ((j & 3) != 3) {
+                TIn::load2(Sb, ((j - (j >> 2)) * G1::Ls + lo) * W + q, e.x[j * V], e.x[j * V + 1]);
                 fix(j);
             }
         });
         phase ^= 1;
-        if (t < L::NBOX) bulk_wait_read_all();                // the previous tile's stores have read the output image
-        __syncthreads();                                      // staging buffer consumed; exchange buffer free
+        if constexpr (!PROGRESSIVE) {
+            if (t < STORE_THREADS) bulk_wait_read_all();      // the previous tile's stores have read the output image
+        }
+        __syncthreads();                                      // staging buffer consumed (and the exchange buffer free)
         if (t == 0 && next < a.tiles) {
             issue(next);
             in_flight = 1;
         }
-        e.template dif<false>(X, a.tw);
+        if constexpr (PROGRESSIVE) {
+            e.template compute<1, false>(a.tw);
+            if (t < STORE_THREADS) bulk_wait_read_all();
+            __syncthreads();                                  // exchange buffer free
+            e.template smem_rw<1, true>(X);
+            __syncthreads();
+            e.template smem_rw<2, false>(X);
+            static_for<2, S>([&](auto s_) {
+                constexpr int s = decltype(s_)::value;
+                if constexpr (Engine<C>::template fused_write_ok<s>()) {
+                    e.template compute_and_write<s>(X, a.tw);
+                } else {
+                    e.template compute<s, false>(a.tw);
+                    e.template smem_rw<s, true>(X);
+                }
+                __syncthreads();
+                e.template smem_rw<s + 1, false>(X);
+            });
+        } else {
+            e.template dif<false>(X, a.tw);
+        }
         __syncthreads();                                      // the last exchange is consumed: X becomes the output image
         {
-            using GS = Geo<C, S>;
-            constexpr int VS = GS::V, rs = GS::r, KS = N / rs;
-            static_assert(VS == 2 && (rs == 8 || rs == 16 || rs == 32), "one register pair per last-stage slot");
             int b0, qq;
             e.last_index(0, b0, qq);
             const bool scaled = a.scale != 1.0f;
@@ -137,14 +181,26 @@ __global__ void __launch_bounds__(C::THREADS, CPS)
                     pb = make_float2(pb.x * a.scale, pb.y * a.scale);
                 }
                 TOut::store2(X, (k * KS + b0) * W + qq, pa, pb);
+                if constexpr (PROGRESSIVE && k >= 12) {       // outputs arrive as k = c, c + 4, c + 8, c + 12 for c = 0..3
+                    fence_async_smem();
+                    __syncthreads();
+                    if (t < 4) {
+                        const int box = (k - 12) + 4 * t;
+                        tma_store_2d(&tm_out, (int)(tile * XW_OUT), box * L::BOX_ROWS,
+                                     reinterpret_cast<const char*>(X) + box * (L::BOX_ROWS * W * TOut::ELEM_BYTES));
+                        bulk_commit();
+                    }
+                }
             });
         }
-        fence_async_smem();
-        __syncthreads();
-        if (t < L::NBOX) {
-            tma_store_2d(&tm_out, (int)(tile * XW_OUT), t * L::BOX_ROWS,
-                         reinterpret_cast<const char*>(X) + t * (L::BOX_ROWS * W * TOut::ELEM_BYTES));
-            bulk_commit();
+        if constexpr (!PROGRESSIVE) {
+            fence_async_smem();
+            __syncthreads();
+            if (t < L::NBOX) {
+                tma_store_2d(&tm_out, (int)(tile * XW_OUT), t * L::BOX_ROWS,
+                             reinterpret_cast<const char*>(X) + t * (L::BOX_ROWS * W * TOut::ELEM_BYTES));
+                bulk_commit();
+            }
         }
     }
     if (gave_up) {
@@ -154,7 +210,7 @@ __global__ void __launch_bounds__(C::THREADS, CPS)
             if (in_flight) mbar_wait(&bar[0], phase, kDefaultWaitPolls);
         }
     }
-    if (t < L::NBOX) bulk_wait_all();
+    if (t < STORE_THREADS) bulk_wait_all();
 }
 
 // cuTensorMapEncodeTiled through the runtime's driver entry point (no link against libcuda)
