@@ -23,9 +23,10 @@ namespace b200fft {
 // per multiprocessor, i.e. boxes with 16-byte rows (144 us); two warp groups of two columns each that take
 // turns on one 64 KiB exchange buffer, so that one group computes while the other exchanges, with the whole
 // next tile staged (76 us, the same with the 32-byte swizzle against the bank conflicts of its half-row
-// accesses, and 74 us on contiguous tiles moved as 64 KiB boxes: the time is set by the traffic through shared
-// memory, about 1 MiB per 128 KiB tile with the staging on both ends, not by the access pattern in main
-// memory). Every wait is bounded: a CTA whose wait runs out raises
+// accesses, and 74 us on contiguous tiles moved as 64 KiB boxes: the access pattern in main memory is not what
+// sets the time; a second form of it that spends the freed 64 KiB on half of the output image, so that the
+// stores need not be read out before the next exchange, took 89 us: its plain-load quarter touches 32 cache
+// lines per warp-level load). Every wait is bounded: a CTA whose wait runs out raises
 // g_tma_timeouts once, stops taking tiles, waits (bounded again) for the copies it still has in flight
 // and returns; the output of that call is then incomplete.
 __device__ int g_tma_timeouts = 0;   // CTAs whose wait for a copy ran out of polls (never expected)
