@@ -242,7 +242,9 @@ int sar_rda_set_workspace(sar_rda_params_t params, void *device_ptr, size_t byte
 /* Variant choice; every form gives the same image to rounding.
  *   "fused_rcmc"   1 runs step 2 as the single fused kernel (RCMC + filter + inverse azimuth FFT on
  *                  column tiles: three passes over memory in all, the paper's best form); 0 runs it as a
- *                  row pass followed by the inverse column FFT (four passes, but faster on B200; the
+ *                  row pass followed by the inverse column FFT (four passes, but faster on B200; with fp16
+ *                  intermediates and 4096 pulses the row pass writes a second fp16 image, one more rounding,
+ *                  else the complex64 output on which the column pass then runs in place; the
  *                  default whenever the scene allows it: B200FFT_ERR_UNSUPPORTED if the migration grows
  *                  by more than 48 bins over 1024 range bins or n_range is not a multiple of 1024).
  *   "layout"       0 (default) keeps the intermediate image row-major and transforms its columns

@@ -267,17 +267,18 @@ cudaError_t launch_cols_stream(const FftArgs& a, cudaStream_t st) {
     g_launch_count.fetch_add(1, std::memory_order_relaxed);
     return cudaGetLastError();
 }
-template <class C, bool INV, class TS, int CPS = 1>
+template <class C, bool INV, class TS, class TO = TS, int CPS = 1>
 constexpr KernelEntry make_stream_entry() {
     return KernelEntry{C::N, C::W, C::G, 1, C::THREADS, Stream<C, TS, CPS>::SMEM_BYTES, C::TW_TOTAL,
                        VAR_STREAM, INV,
-                       TS::ELEM_BYTES == 8 ? 0 : 1, TS::ELEM_BYTES == 8 ? 0 : 1,
-                       &launch_cols_stream<C, INV, TS, TS, CPS>, &launch_build_tw<C>};
+                       TS::ELEM_BYTES == 8 ? 0 : 1, TO::ELEM_BYTES == 8 ? 0 : 1,
+                       &launch_cols_stream<C, INV, TS, TO, CPS>, &launch_build_tw<C>};
 }
 static const KernelEntry k_cols_stream[] = {
     make_stream_entry<T4096, false, StoreC64>(), make_stream_entry<T4096, true, StoreC64>(),
     make_stream_entry<T4096, false, StoreC32H>(), make_stream_entry<T4096, true, StoreC32H>(),
     make_stream_entry<T2048, false, StoreC64>(), make_stream_entry<T2048, true, StoreC64>(),
+    make_stream_entry<T4096, true, StoreC32H, StoreC64>(),    // SAR with fp16 intermediates: the last pass writes the complex64 image
 };
 
 int tma_timeouts() {

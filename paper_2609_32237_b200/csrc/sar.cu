@@ -326,7 +326,7 @@ struct RcmcRows {
     static constexpr int TPB = 256;
 };
 
-template <class TIn>
+template <class TIn, class TOut = StoreC64>
 __global__ void __launch_bounds__(RcmcRows::TPB) sar_rcmc_filter_rows_kernel(const SarArgs a, int chunks) {
     constexpr int COLS = RcmcRows::COLS, HALO = RcmcRows::HALO, TPB = RcmcRows::TPB;
     constexpr int EB = TIn::ELEM_BYTES, GRAN = 16 / EB;
@@ -349,7 +349,7 @@ __global__ void __launch_bounds__(RcmcRows::TPB) sar_rcmc_filter_rows_kernel(con
         *reinterpret_cast<uint4*>(srow + i * GRAN) = v;
     }
     __syncthreads();
-    float2* out = reinterpret_cast<float2*>(a.out) + (int64_t)k * a.ld;
+    const int64_t orow = (int64_t)k * a.ld;
     const float g = mg.x + mg.y;
 #pragma unroll
     for (int h = 0; h < COLS / (2 * TPB); ++h) {
@@ -394,7 +394,7 @@ __global__ void __launch_bounds__(RcmcRows::TPB) sar_rcmc_filter_rows_kernel(con
         const float2 fa = filter_phase(ph, n);
         const float2 fb = cmul(fa, step);
         const float2 ya = cmul(sa, fa), yb = cmul(sb, fb);
-        *reinterpret_cast<float4*>(out + n) = make_float4(ya.x, ya.y, yb.x, yb.y);
+        TOut::store2(a.out, orow + n, ya, yb);
     }
 }
 
@@ -699,6 +699,7 @@ struct b200fft_sar_s {
     const KernelEntry* azfft;
     const SarEntry* rcmc;
     const KernelEntry* azifft;   // in-place inverse column transform of the unfused variant
+    const KernelEntry* azifft_h; // fp16 intermediates: inverse column transform from an fp16 image to the complex64 output
     bool can_unfuse;
     // slab intermediate ("layout" 1)
     const SarEntry* range_slab;
@@ -781,6 +782,11 @@ extern "C" int sar_rda_params_create(sar_rda_params_t* params, const sar_rda_des
     p->rcmc = find(k_rcmc, na, dt, false);
     p->rcmc_slab = find(k_rcmc, na, dt, true);
     p->azifft = cols_kernel(true, B200FFT_C64);
+    p->azifft_h = nullptr;
+    if (dt == B200FFT_C32H && nr / 4 > sms) {
+        const KernelEntry* k = find_cols_kernel(na, true, B200FFT_C32H, B200FFT_C64, 0, VAR_STREAM);
+        if (k && nr % k->w == 0 && k->tw_total == p->rcmc->tw_total) p->azifft_h = k;
+    }
     for (int i = 0; i < 2; ++i) {
         p->azfft_slab[i] = find_sar_cols_kernel(na, 2 << i, false, dt, dt);
         p->azifft_slab[i] = find_sar_cols_kernel(na, 2 << i, true, dt, B200FFT_C64);
@@ -959,15 +965,24 @@ extern "C" int sar_rda_run_step(const void* raw, sar_rda_params_t p, void* out, 
         return ok(k->launch(f, st));
     }
     const int chunks = (int)(nr / RcmcRows::COLS);
-    if (dt == B200FFT_C64)
+    // With fp16 intermediates the row pass writes a second fp16 image (one more rounding, as in the paper's
+    // four-pass accounting of 40 bytes per pixel) where the inverse column kernel for it is compiled; else the
+    // complex64 output image, on which the inverse column pass then runs in place.
+    const bool half_image = dt == B200FFT_C32H && p->azifft_h != nullptr;
+    if (dt == B200FFT_C64) {
         sar_rcmc_filter_rows_kernel<StoreC64><<<(unsigned)(na * chunks), RcmcRows::TPB, 0, st>>>(a, chunks);
-    else
+    } else if (half_image) {
+        a.out = buf1;
+        sar_rcmc_filter_rows_kernel<StoreC32H, StoreC32H><<<(unsigned)(na * chunks), RcmcRows::TPB, 0, st>>>(a, chunks);
+    } else {
         sar_rcmc_filter_rows_kernel<StoreC32H><<<(unsigned)(na * chunks), RcmcRows::TPB, 0, st>>>(a, chunks);
+    }
     g_launch_count.fetch_add(1, std::memory_order_relaxed);
     if (cudaGetLastError() != cudaSuccess) return B200FFT_ERR_CUDA;
-    f.in = out; f.out = out;
-    f.tiles = nr / p->azifft->w; f.dist = nr;
-    return ok(p->azifft->launch(f, st));
+    const KernelEntry* inv = half_image ? p->azifft_h : p->azifft;
+    f.in = half_image ? buf1 : out; f.out = out;
+    f.tiles = nr / inv->w; f.dist = nr;
+    return ok(inv->launch(f, st));
 }
 
 extern "C" int sar_rda_set_option(sar_rda_params_t p, const char* key, int64_t value) {

@@ -33,6 +33,11 @@ def test_noalloc_matches_the_plan_path_twice_in_a_row():
         want = oracle.fft_rows(x.astype(np.complex128), direction)
         worst, pooled = worst_rel_l2(got.cpu().numpy(), want)
         assert worst <= 1e-5 and pooled <= 1e-5
+        # in place (the header allows in == out: the first pass has read the input before the second writes)
+        same = d.clone()
+        B.fft_execute_noalloc(n, batch, direction, same.data_ptr(), same.data_ptr(), st)
+        torch.cuda.synchronize()
+        assert bool((same == got).all())
 
     # sizes beyond the fixed scratch are refused with a clear status, not run
     big = torch.zeros(2 * B.NOALLOC_MAX_ELEMS, dtype=torch.complex64, device="cuda")
