@@ -231,6 +231,22 @@ def full_scene():
     return sc, raw, img
 
 
+def test_wide_swath_frame():
+    """1024 pulses x 8192 range samples: the 8192-point range compression kernel and 128 chunks of the row
+    pass, both intermediate types, row-major and slab layouts."""
+    sc = inputs.x_band_scene(n_azimuth=1024, n_range=8192, n_targets=0)
+    sc.antenna_m = 3.0
+    sc.targets = inputs.seeded_target_cells(sc, 4, seed=21)
+    raw = inputs.simulate_raw(sc, seed=21)
+    img = oracle.sar_rda(oracle.sar_params(sc), raw)
+    for dtype, tol in ((C64, 1e-5), (C32H, 5e-3)):
+        for layout in (0, 1):
+            got = _gpu_chain(sc, raw, dtype, layout=layout)
+            assert rel_l2(got, img) <= tol
+            for cell in sc.targets:
+                assert quality.peak_cell(got, tuple(cell)) == tuple(cell)
+
+
 def test_other_frame_sizes_and_error_paths():
     """A 2048 x 1024 frame with a 5 us pulse (other kernel instantiations), both intermediate
     types and both forms of step 2; then the host-side error paths of the SAR calls."""
