@@ -351,6 +351,16 @@ def bench_fft(torch, B, n, batch, dtype, seed, steps, warmup, layout="rows", dir
     return total, per, clean_per
 
 
+def issue_roofline(key, ms):
+    """For the workloads bound by instruction issue: the warp instructions of one launch (from the ncu capture
+    summarised under profiles/) against what the GPU can issue in the measured time at its maximum clock."""
+    inst = metrics.NCU_WARP_INSTRUCTIONS[key]
+    floor_ms = metrics.issue_roof_seconds(inst) * 1e3
+    return {"bound": "alu", "unit": "warp instructions/s", "achieved": inst / (ms * 1e-3),
+            "peak": 148 * 4 * 1.965e9, "frac": floor_ms / ms, "warp_instructions": inst, "ms_at_peak": floor_ms,
+            "note": "peak = 148 SMs x 4 schedulers x 1.965 GHz, one warp instruction per scheduler and cycle"}
+
+
 def summarize(per_ms, nbytes, peak):
     med = float(np.median(per_ms))
     q1, q3 = np.percentile(per_ms, [25, 75])
@@ -558,6 +568,8 @@ def run_others(torch, B, args, peak):
     fft_case("fft_n16384_b8192_c64", 16384, 8192, 0, 2)
     fft_case("fft_n8192_b16384_c32h", 8192, 16384, 1, 2)
     fft_case("fft_n16384_b8192_c32h", 16384, 8192, 1, 2)
+    for name, key in (("fft_n8192_b16384_c32h", "fft_rows_8192_b16384_c32h"), ("fft_n16384_b8192_c32h", "fft_rows_16384_b8192_c32h")):
+        out[name]["issue_roofline"] = issue_roofline(key, out[name]["ms_median"])
     fft_case("fft_n1024_b256_c64", 1024, 256, 0, 0)
 
     # block floating point on fp16 storage (one exponent per transform): the cost of the maximum search
@@ -632,6 +644,8 @@ def run_others(torch, B, args, peak):
             r = summarize(per, metrics.sar_bytes(4096, 4096, dtype), peak)
             r["ms_per_image"] = r["ms_median"]
             r["options"] = opts
+            if not suffix:
+                r["issue_roofline"] = issue_roofline("sar_4096x4096_fp32" if dtype == 0 else "sar_4096x4096_fp16", r["ms_median"])
             per_step = [time_cold(torch, (lambda s=s: B.sar_rda_run_step(rd.data_ptr(), p, img.data_ptr(), s, stream.cuda_stream)),
                                   stream, scratch, steps, 1) for s in range(3)]
             r["passes_ms"] = {"range_compression": float(np.median(per_step[0])),

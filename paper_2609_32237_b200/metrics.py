@@ -16,6 +16,22 @@ BYTES_PER_POINT = {0: 16, 1: 8}        # storage dtype -> bytes in + bytes out p
 NCU_TRAFFIC_BYTES = {"fft_rows_4096_c64": 2095526000}
 
 
+# smsp__inst_executed.sum (warp instructions) per launch or per image from the same captures, for the
+# workloads whose roof is instruction issue rather than HBM
+NCU_WARP_INSTRUCTIONS = {
+    "fft_rows_8192_b16384_c32h": 247463936,
+    "fft_rows_16384_b8192_c32h": 266299384,
+    "sar_4096x4096_fp32": 54689792 + 27472854 + 59949056 + 27695506,
+    "sar_4096x4096_fp16": 55210000 + 28980000 + 66140000 + 27700000,
+}
+
+
+def issue_roof_seconds(warp_instructions: float, sms: int = 148, schedulers_per_sm: int = 4, sm_mhz: float = 1965.0) -> float:
+    """Shortest time in which one GPU can issue that many warp instructions: every scheduler of every
+    multiprocessor issues at most one per cycle."""
+    return warp_instructions / (sms * schedulers_per_sm * sm_mhz * 1e6)
+
+
 def fft_flops(n: int, batch: int = 1) -> float:
     return 5.0 * n * math.log2(n) * batch
 

@@ -25,3 +25,11 @@ def test_footprints():
     assert metrics.fft_bytes(8192, 16384, 1) == 1024 ** 3
     assert metrics.sar_bytes(4096, 4096, 0) == 48 * 4096 * 4096
     assert metrics.sar_bytes(4096, 4096, 1) == 32 * 4096 * 4096
+
+
+def test_issue_roof_arithmetic():
+    # 148 multiprocessors x 4 schedulers x 1.965 GHz = 1.163e12 warp instructions per second
+    assert abs(metrics.issue_roof_seconds(1.16328e12) - 1.0) < 1e-6
+    # the fp16-storage transform of N = 8192 needs 213 us of issue slots against 164 us of HBM time
+    t = metrics.issue_roof_seconds(metrics.NCU_WARP_INSTRUCTIONS["fft_rows_8192_b16384_c32h"])
+    assert 2.1e-4 < t < 2.15e-4 and t > metrics.fft_bytes(8192, 16384, 1) / 6532.2e9
