@@ -56,7 +56,7 @@ typedef struct b200fft_sar_s *sar_rda_params_t;
  *   columns  dist == 1, stride >= batch, stride and batch even: the columns of
  *            a row-major matrix (paper, Section "End to End": the FFT that
  *            reads the columns directly)
- * Supported sizes: n a power of two, 32 <= n <= 32768 in a single pass over
+ * Supported sizes: n a power of two, 8 <= n <= 32768 in a single pass over
  * memory (columns: 64 <= n <= 8192; rows of n = 32768 on a cluster of two
  * thread blocks that share the transform through distributed shared memory);
  * 2^16 <= n <= 2^20 (rows only) by a two-pass four-step split (the paper's

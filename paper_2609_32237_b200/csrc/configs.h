@@ -11,6 +11,9 @@ namespace b200fft {
 using R128 = Cfg<128, 1, 16, 16, 1, 16, 8>;
 using R64 = Cfg<64, 1, 16, 32, 1, 8, 8>;
 using R32 = Cfg<32, 1, 16, 64, 1, 4, 8>;
+// below the paper's range: one thread per transform (16 = 4 x 4, 8 = 2 x 4), 128 transforms per CTA
+using R16 = Cfg<16, 1, 16, 128, 1, 4, 4>;
+using R8 = Cfg<8, 1, 8, 128, 1, 2, 4>;
 using R256 = Cfg<256, 1, 32, 16, 1, 16, 16>;
 using R512 = Cfg<512, 1, 32, 8, 1, 16, 32>;
 using R1024 = Cfg<1024, 1, 32, 4, 1, 32, 32>;

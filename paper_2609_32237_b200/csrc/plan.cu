@@ -150,7 +150,7 @@ extern "C" int fft_plan_create(fft_plan_t* plan, int64_t n, int64_t batch, int64
     if (direction != B200FFT_FORWARD && direction != B200FFT_INVERSE) return B200FFT_ERR_INVALID_ARG;
     if (storage_dtype != B200FFT_C64 && storage_dtype != B200FFT_C32H) return B200FFT_ERR_INVALID_ARG;
     if (!is_pow2(n)) return B200FFT_ERR_UNSUPPORTED;
-    if (n < 32 || n > (1 << 20)) return B200FFT_ERR_UNSUPPORTED;
+    if (n < 8 || n > (1 << 20)) return B200FFT_ERR_UNSUPPORTED;
 
     Layout layout;
     if (stride == 1 && dist >= n) layout = LAYOUT_ROWS;

@@ -425,10 +425,10 @@ def test_seeded_random_plans_against_the_oracle():
         assert worst <= tol and pooled <= tol, (trial, layout, n, dtype, direction, worst)
 
 
-@pytest.mark.parametrize("n", [32, 64, 128])
+@pytest.mark.parametrize("n", [8, 16, 32, 64, 128])
 def test_small_transforms(n):
-    """N = 32, 64, 128: several transforms per CTA, ragged batches, both directions, padding,
-    fp16 storage; each against the direct DFT."""
+    """N = 8 ... 128: several transforms per CTA (one thread per transform at N = 8 and 16), ragged
+    batches, both directions, padding, fp16 storage; each against the direct DFT."""
     for batch in (1, 5, 130, 1000):
         _check_rows(n, batch, seed=300 + n + batch, gaussian=(batch == 130))
         _check_rows(n, batch, seed=301 + n + batch, direction=INV)
