@@ -43,7 +43,7 @@ def test_bad_arguments_are_rejected_on_the_host(B):
     assert L.fft_plan_create(ctypes.byref(h), 1024, 1, 1, 1024, 0, 0) == 1       # direction
     assert L.fft_plan_create(ctypes.byref(h), 1024, 1, 1, 1024, -1, 7) == 1      # dtype
     assert L.fft_plan_create(ctypes.byref(h), 1000, 1, 1, 1000, -1, 0) == 2      # not a power of two
-    assert L.fft_plan_create(ctypes.byref(h), 16, 1, 1, 16, -1, 0) == 2          # too small
+    assert L.fft_plan_create(ctypes.byref(h), 4, 1, 1, 4, -1, 0) == 2            # too small
     assert L.fft_plan_create(ctypes.byref(h), 1 << 21, 1, 1, 1 << 21, -1, 0) == 2
     assert L.fft_plan_create(ctypes.byref(h), 1024, 4, 3, 7, -1, 0) == 2         # layout class
     assert L.fft_plan_create(ctypes.byref(h), 1024, 4, 1, 1025, -1, 0) == 3      # odd dist
