@@ -294,3 +294,61 @@ def test_other_frame_sizes_and_error_paths():
     with pytest.raises(B.B200FftError) as e:
         B.sar_rda_params_create(bad)
     assert e.value.status == 2
+
+
+def _noise_frame(n_azimuth, n_range, seed):
+    g = np.random.default_rng(seed)
+    return (g.standard_normal((n_azimuth, n_range)) + 1j * g.standard_normal((n_azimuth, n_range))).astype(np.complex64)
+
+
+@pytest.mark.parametrize("prf_hz,row_pass", [(986.0, True), (987.0, False), (1660.0, False)])
+def test_shift_growth_at_the_edge_of_the_row_pass_guard(prf_hz, row_pass):
+    """The row pass of step 2 stages 1024 + 64 range samples per CTA and is offered only while the
+    integer shift grows by at most 48 bins over 1024 range bins at the Doppler edge. With a 0.24 m
+    wavelength at 200 m/s that growth is 47.97 bins at PRF 986 Hz (accepted; shifts reach ~800 bins)
+    and 48.08 at 987 Hz (refused: step 2 falls back to the fused column kernel); 1660 Hz sits just
+    below the largest PRF the calls accept at all (shifts beyond the swath width). White noise as
+    the raw frame makes every output pixel depend on the window it was read from."""
+    from paper_2609_32237_b200 import binding as B
+    sc = inputs.l_band_scene(n_azimuth=1024, n_range=2048, targets=[])
+    sc.prf_hz = prf_hz
+    raw = _noise_frame(1024, 2048, seed=int(prf_hz))
+    img = oracle.sar_rda(oracle.sar_params(sc), raw)
+    assert np.abs(img).max() > 0
+    p = B.sar_rda_params_create(B.sar_desc_from_scene(sc, C64))
+    try:
+        if row_pass:
+            B.sar_rda_set_option(p, "fused_rcmc", 0)
+        else:
+            with pytest.raises(B.B200FftError) as e:
+                B.sar_rda_set_option(p, "fused_rcmc", 0)
+            assert e.value.status == 2
+    finally:
+        B.sar_rda_params_destroy(p)
+    for dtype, tol in ((C64, 1e-5), (C32H, 5e-3)):
+        assert rel_l2(_gpu_chain(sc, raw, dtype), img) <= tol                   # the default form
+        assert rel_l2(_gpu_chain(sc, raw, dtype, fused=True), img) <= tol
+
+
+@pytest.mark.parametrize("prf_hz,accepted", [(410.0, True), (415.0, False)])
+def test_shift_spread_at_the_edge_of_the_slab_guard(prf_hz, accepted):
+    """The slab-layout row pass holds 32 Doppler bins x 64 range bins per CTA and is offered only
+    while the integer shift spreads by at most 16 bins inside one CTA: 15.9 at PRF 410 Hz, 16.3 at
+    415 Hz for this 1024 x 2048 frame."""
+    from paper_2609_32237_b200 import binding as B
+    sc = inputs.l_band_scene(n_azimuth=1024, n_range=2048, targets=[])
+    sc.prf_hz = prf_hz
+    raw = _noise_frame(1024, 2048, seed=int(prf_hz))
+    if not accepted:
+        p = B.sar_rda_params_create(B.sar_desc_from_scene(sc, C64))
+        try:
+            with pytest.raises(B.B200FftError) as e:
+                B.sar_rda_set_option(p, "layout", 1)
+            assert e.value.status == 2
+        finally:
+            B.sar_rda_params_destroy(p)
+        return
+    img = oracle.sar_rda(oracle.sar_params(sc), raw)
+    for dtype, tol in ((C64, 1e-5), (C32H, 5e-3)):
+        for tile_columns in (2, 4):
+            assert rel_l2(_gpu_chain(sc, raw, dtype, layout=1, tile_columns=tile_columns), img) <= tol
