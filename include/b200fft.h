@@ -106,6 +106,10 @@ int fft_plan_destroy(fft_plan_t plan);
  * B200FFT_ERR_UNSUPPORTED and leaves the plan as it was. Call before set_workspace.
  *   "four_step"  1 routes a rows plan of any supported n >= 4096 through the two-pass split; 0 brings a
  *                plan of n <= 32768 back to its single pass.
+ *   "split_n1"   two-pass plans only: factor n = n1 * n2 with this n1 (a power of two, 64 <= n1 <= 1024,
+ *                64 <= n2 <= 4096; 0 = the default, n1 = 256 for n >= 65536 and the near-square split
+ *                with n1 >= n2 below). Pass 1 transforms the n2 columns of length n1, pass 2 the n1 rows
+ *                of length n2.
  *   "cluster"    c = 1, 2 or 4 (0 = the default rules; other values are B200FFT_ERR_INVALID_ARG): the
  *                single-pass variant in which c CTAs of one thread-block cluster share a tile through
  *                distributed shared memory. Defaults: rows of n = 16384 / 8192 with at most 32 / 16

@@ -62,7 +62,7 @@ __global__ void __launch_bounds__(C::THREADS, C::MINB) fourstep_pass1_kernel(con
     using G = Geo<C, C::S>;
     constexpr int V = G::V, r = G::r, KS = C::N / r;
     static_assert(V >= 2, "register pairs");
-    // k1 < n1 <= 1024 and j2 < n2 <= 1024: the products fit 32 bits
+    // k1 < n1 <= 1024, j2 < n2 and n1 * n2 <= 2^20: the products fit 32 bits
     const unsigned nmask = (unsigned)(a.n - 1), n2 = (unsigned)a.n2;
     const int64_t obase = b * a.dist_out;
     auto twiddle_and_store = [&](auto v_, auto j_, float2 pa, float2 pb) {
@@ -149,7 +149,8 @@ constexpr FourStepEntry make_fs_entry() {
 static const FourStepEntry k_pass1[] = {FS_ENTRIES(F64, 1), FS_ENTRIES(F128, 1), FS_ENTRIES(F256, 1),
                                         FS_ENTRIES(F512, 1), FS_ENTRIES(F1024, 1)};
 static const FourStepEntry k_pass2[] = {FS_ENTRIES(T64, 2), FS_ENTRIES(T128, 2), FS_ENTRIES(T256, 2),
-                                        FS_ENTRIES(T512, 2), FS_ENTRIES(T1024, 2)};
+                                        FS_ENTRIES(T512, 2), FS_ENTRIES(T1024, 2), FS_ENTRIES(T2048, 2),
+                                        FS_ENTRIES(T4096, 2)};
 
 template <size_t K>
 static const FourStepEntry* find(const FourStepEntry (&tab)[K], int n, bool inv, int dtype) {
@@ -168,6 +169,25 @@ __global__ void build_factor_table(float2* tab, int count, int64_t step, int64_t
     tab[i] = make_float2((float)cs, (float)sn);
 }
 
+// n = n1 * n2. Default: n1 = 256 from n = 65536 on (pass 1 then runs on 32 KiB tiles, four CTAs per SM, and
+// pass 2 carries the long transform along contiguous rows; measured for 512 MiB of complex64: 2^17 404 -> 394 us,
+// 2^18 428 -> 402, 2^19 480 -> 441, 2^20 492 -> 476 against the near-square split), the near-square split with
+// n1 >= n2 below. `n1_request` > 0 asks for another one (64 <= n1 <= 1024, 64 <= n2 <= 4096).
+static int fourstep_split(int64_t n, int64_t n1_request, int64_t* n1, int64_t* n2) {
+    int lg = 0;
+    while (((int64_t)1 << lg) < n) ++lg;
+    if (((int64_t)1 << lg) != n || lg < 12 || lg > 20) return B200FFT_ERR_UNSUPPORTED;
+    *n1 = lg >= 16 ? 256 : (int64_t)1 << ((lg + 1) / 2);
+    if (n1_request > 0) {
+        if ((n1_request & (n1_request - 1)) || n1_request < 64 || n1_request > 1024 || n / n1_request < 64 ||
+            n / n1_request > 4096)
+            return B200FFT_ERR_UNSUPPORTED;
+        *n1 = n1_request;
+    }
+    *n2 = n / *n1;
+    return B200FFT_OK;
+}
+
 void fourstep_release(FourStep* fs) {
     if (fs->tw1) cudaFree(fs->tw1);
     if (fs->tw2) cudaFree(fs->tw2);
@@ -176,14 +196,14 @@ void fourstep_release(FourStep* fs) {
     *fs = FourStep();
 }
 
-int fourstep_build(FourStep* fs, int64_t n, int64_t batch, int64_t dist, int direction, int dtype) {
+int fourstep_build(FourStep* fs, int64_t n, int64_t batch, int64_t dist, int direction, int dtype, int64_t n1_request) {
     fourstep_release(fs);
-    int lg = 0;
-    while (((int64_t)1 << lg) < n) ++lg;
-    if (((int64_t)1 << lg) != n || lg < 12 || lg > 20) return B200FFT_ERR_UNSUPPORTED;
+    int64_t n1, n2;
+    const int rc = fourstep_split(n, n1_request, &n1, &n2);
+    if (rc != B200FFT_OK) return rc;
     fs->n = n;
-    fs->n1 = (int64_t)1 << ((lg + 1) / 2);
-    fs->n2 = n / fs->n1;
+    fs->n1 = n1;
+    fs->n2 = n2;
     fs->batch = batch;
     fs->dist = dist;
     fs->direction = direction;
@@ -213,18 +233,9 @@ int fourstep_build(FourStep* fs, int64_t n, int64_t batch, int64_t dist, int dir
     return B200FFT_OK;
 }
 
-static int fourstep_split(int64_t n, int64_t* n1, int64_t* n2) {
-    int lg = 0;
-    while (((int64_t)1 << lg) < n) ++lg;
-    if (((int64_t)1 << lg) != n || lg < 12 || lg > 20) return B200FFT_ERR_UNSUPPORTED;
-    *n1 = (int64_t)1 << ((lg + 1) / 2);
-    *n2 = n / *n1;
-    return B200FFT_OK;
-}
-
 size_t fourstep_table_elems(int64_t n, int direction, int dtype) {
     int64_t n1, n2;
-    if (fourstep_split(n, &n1, &n2) != B200FFT_OK) return 0;
+    if (fourstep_split(n, 0, &n1, &n2) != B200FFT_OK) return 0;
     const bool inv = direction == B200FFT_INVERSE;
     const FourStepEntry* p1 = find(k_pass1, (int)n1, inv, dtype);
     const FourStepEntry* p2 = find(k_pass2, (int)n2, inv, dtype);
@@ -238,7 +249,7 @@ int fourstep_build_in_place(FourStep* fs, int64_t n, int64_t batch, int64_t dist
                             float2* tables, size_t table_elems, cudaStream_t st) {
     *fs = FourStep();
     int64_t n1, n2;
-    int rc = fourstep_split(n, &n1, &n2);
+    int rc = fourstep_split(n, 0, &n1, &n2);
     if (rc != B200FFT_OK) return rc;
     const size_t need = fourstep_table_elems(n, direction, dtype);
     if (need == 0) return B200FFT_ERR_UNSUPPORTED;

@@ -18,7 +18,9 @@ struct FourStep {
     float2* tw_hi = nullptr;                // exp(-2 pi i 1024 m / n), m = 0..n/1024-1
 };
 
-int fourstep_build(FourStep* fs, int64_t n, int64_t batch, int64_t dist, int direction, int dtype);
+// n1_request = 0: the default split; otherwise n = n1_request * n2 if both passes exist for it.
+int fourstep_build(FourStep* fs, int64_t n, int64_t batch, int64_t dist, int direction, int dtype,
+                   int64_t n1_request = 0);
 int fourstep_execute(const FourStep* fs, const void* in, void* out, void* workspace, cudaStream_t st);
 void fourstep_release(FourStep* fs);
 

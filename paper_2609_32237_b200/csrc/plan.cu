@@ -212,6 +212,15 @@ extern "C" int fft_plan_set_option(fft_plan_t p, const char* key, int64_t value)
         }
         return B200FFT_OK;
     }
+    if (std::strcmp(key, "split_n1") == 0) {       // two-pass plans: n = n1 * n2 with this n1 (0 = the default split)
+        if (!p->four_step || value < 0) return B200FFT_ERR_UNSUPPORTED;
+        FourStep fs;
+        int rc = fourstep_build(&fs, p->n, p->batch, p->dist, p->direction, p->dtype, value);
+        if (rc != B200FFT_OK) return rc;
+        fourstep_release(&p->fs);
+        p->fs = fs;
+        return B200FFT_OK;
+    }
     if (std::strcmp(key, "prefetch") == 0) {
         if (value < -1 || value > (1 << 20)) return B200FFT_ERR_INVALID_ARG;
         p->prefetch_ahead = (int)value;

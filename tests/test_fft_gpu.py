@@ -193,12 +193,32 @@ def test_four_step_forced_at_single_pass_sizes(n, direction):
     _check_rows(n, 5, seed=41, direction=direction, options={"four_step": 1})
 
 
-@pytest.mark.parametrize("lg", [15, 16, 17, 18, 20])
+@pytest.mark.parametrize("lg", [15, 16, 17, 18, 19, 20])
 def test_four_step_large(lg):
     n = 1 << lg
     batch = 3 if lg < 20 else 2
     _check_rows(n, batch, seed=50 + lg, gaussian=True)
     _check_rows(n, batch, seed=60 + lg, direction=INV)
+
+
+@pytest.mark.parametrize("lg,n1", [(16, 64), (16, 1024), (17, 128), (17, 512), (18, 64), (18, 1024),
+                                   (19, 128), (19, 1024), (20, 512), (20, 1024)])
+def test_four_step_other_splits(lg, n1):
+    """n = n1 * n2 with a requested n1 (option split_n1) instead of the default: every pass-1 length
+    64..1024 and every pass-2 length 64..4096 occurs once; a split without kernels is refused."""
+    from paper_2609_32237_b200 import binding as B
+    n = 1 << lg
+    _check_rows(n, 2, seed=80 + lg, gaussian=True, options={"four_step": 1, "split_n1": n1})
+    _check_rows(n, 2, seed=90 + lg, direction=INV, options={"four_step": 1, "split_n1": n1})
+    if lg == 20:
+        plan = B.fft_plan_create(n, 2, 1, n, FWD, C64)
+        try:
+            for bad in (128, 96, 2048):          # n2 = 8192 has no pass 2; not a power of two; n1 too long
+                with pytest.raises(B.B200FftError) as e:
+                    B.fft_plan_set_option(plan, "split_n1", bad)
+                assert e.value.status == 2
+        finally:
+            B.fft_plan_destroy(plan)
 
 
 def test_four_step_fp16_and_workspace_errors():
