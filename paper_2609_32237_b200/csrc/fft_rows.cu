@@ -193,7 +193,7 @@ const KernelEntry* find_rows_kernel(int n, bool inverse, int in_dtype, int out_d
         return nullptr;
     }
     if (variant == VAR_PLAIN && cl == 0) cl = default_cluster(n, batch);
-    const EntryList lists[3] = {rows_entries_small(), rows_entries_large(), rows_entries_cluster()};
+    const EntryList lists[4] = {rows_entries_small(), rows_entries_large(), rows_entries_cluster(), rows_entries_tiny()};
     for (const EntryList& l : lists)
         for (int i = 0; i < l.count; ++i) {
             const KernelEntry& e = l.first[i];

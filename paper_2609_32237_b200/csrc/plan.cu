@@ -61,6 +61,9 @@ static int build_single_pass(b200fft_plan_s* p) {
         // only half of the tile can wait beside the exchange buffer), so there it is only taken on request.
         const bool by_default = p->n == 16384 && p->dtype == B200FFT_C32H && p->batch >= 2 * (int64_t)p->sms;
         if (p->staged == 1 || (p->staged == -1 && by_default)) variant = VAR_STAGED;
+        // Transforms of at most 32 points packed back to back: the chunk-staging kernel (measured for 1 GiB of
+        // complex64 in and out, against the plain kernel: see the option's note in the header).
+        if (p->n <= 32 && p->dist == p->n && p->staged != 0) variant = VAR_TINY;
     }
     if (p->layout == LAYOUT_COLS && variant == VAR_PLAIN && cl == 0) {
         // default rules, widest first: 16-column tiles for n <= 1024 where they divide the batch ...

@@ -20,6 +20,7 @@ enum Variant : int {
     VAR_STREAM,          // columns: persistent kernel, tiles staged in and out by the tensor memory accelerator
     VAR_WIDE,            // columns: tiles wider than four columns on one CTA
     VAR_WIDE_CLUSTER,    // columns: tiles of 32768 / n columns shared by a cluster of two CTAs
+    VAR_TINY,            // rows, n <= 32, contiguous batch: one thread per transform, chunk staged through shared memory
 };
 
 struct KernelEntry {
@@ -112,7 +113,8 @@ struct EntryList {
     const KernelEntry* first;
     int count;
 };
-EntryList rows_entries_small();     // N = 32 .. 2048
+EntryList rows_entries_small();     // N = 8 .. 2048
+EntryList rows_entries_tiny();      // N = 8 .. 32, contiguous batches
 EntryList rows_entries_large();     // N = 4096 .. 16384 and the alternative factorisations
 EntryList rows_entries_cluster();   // transforms shared by a cluster of CTAs
 EntryList cols_entries_more();      // column tiles on clusters, wide column tiles

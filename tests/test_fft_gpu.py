@@ -460,6 +460,27 @@ def test_small_transforms(n):
     assert max(worst_rel_l2(got, want)) <= TOL16
 
 
+@pytest.mark.parametrize("n", [8, 16, 32])
+def test_tiny_transforms_both_kernels(n):
+    """N <= 32 on a contiguous batch runs the chunk-staging kernel by default (one thread per transform,
+    128 transforms per CTA through shared memory) and the plain kernel with staged = 0: both against the
+    direct DFT, batches that end inside a CTA's chunk, in place, both directions and storage types."""
+    for batch in (1, 127, 128, 129, 1000, 4099):
+        for direction in (FWD, INV):
+            x = inputs.gaussian_complex64((batch, n), 310 + n + batch)
+            want = oracle.fft_rows(x.astype(np.complex128), direction)
+            for options in (None, {"staged": 0}):
+                got = run_fft(to_device_c64(x), n, batch, 1, n, direction, C64, options=options).cpu().numpy()
+                assert max(worst_rel_l2(got, want)) <= TOL32, (n, batch, direction, options)
+            got = run_fft(to_device_c64(x), n, batch, 1, n, direction, C64, inplace=True).cpu().numpy()
+            assert max(worst_rel_l2(got, want)) <= TOL32
+            h = inputs.to_half_storage(x)
+            want16 = oracle.fft_rows(inputs.from_half_storage(h), direction)
+            for options in (None, {"staged": 0}):
+                got = half_to_c128(run_fft(to_device_half(h), n, batch, 1, n, direction, C32H, options=options))
+                assert max(worst_rel_l2(got, want16)) <= TOL16, (n, batch, direction, options)
+
+
 @pytest.mark.parametrize("n,batch", [(16384, 5), (16384, 300), (16384, 449)])
 @pytest.mark.parametrize("dtype", [C64, C32H])
 def test_staged_persistent_rows(n, batch, dtype):
