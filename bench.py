@@ -167,9 +167,10 @@ class ClockSampler:
 
 
 def run_landscape(args):
-    """Throughput against transform size, N = 32 ... 2^20 (the paper's Figure "landscape", our
+    """Throughput against transform size, N = 8 ... 2^20 (the paper's Figure "landscape", our
     kernels only): cold on a 1 GiB footprint (512 MiB in + 512 MiB out, a 512 MiB scratch write
-    before every sample) and hot on a 32 MiB footprint that stays in the 126 MB L2."""
+    before every sample), the same number of points cold with fp16 storage (half the bytes), and
+    hot on a 32 MiB footprint that stays in the 126 MB L2."""
     import torch
     torch.cuda.set_device(0)
     from paper_2609_32237_b200 import binding as B
@@ -179,12 +180,13 @@ def run_landscape(args):
     big = torch.randn(1 << 26, 2, device="cuda")
     big_out = torch.empty_like(big)
     rows = []
-    for lg in range(5, 21):
+    for lg in range(3, 21):
         n = 1 << lg
         row = {"n": n}
-        for label, points, cold in (("cold_1gib", 1 << 26, True), ("hot_32mib", 1 << 21, False)):
+        for label, points, cold, dtype in (("cold_1gib", 1 << 26, True, 0), ("cold_fp16_storage", 1 << 26, True, 1),
+                                           ("hot_32mib", 1 << 21, False, 0)):
             batch = points // n
-            plan = B.fft_plan_create(n, batch, 1, n, -1, 0)
+            plan = B.fft_plan_create(n, batch, 1, n, -1, dtype)
             need = B.fft_plan_workspace_bytes(plan)
             ws = None
             if need:
@@ -194,7 +196,7 @@ def run_landscape(args):
             for _ in range(3):
                 call()
             torch.cuda.synchronize()
-            nb = metrics.fft_bytes(n, batch, 0)
+            nb = metrics.fft_bytes(n, batch, dtype)
             if cold:
                 per = []
                 for _ in range(9):
@@ -220,7 +222,7 @@ def run_landscape(args):
             row[label] = {"batch": batch, "us": ms * 1e3, "gbs": nb / ms / 1e6,
                           "gflops": metrics.fft_gflops(n, batch, ms * 1e-3)}
         rows.append(row)
-    print(json.dumps({"landscape": "complex64 forward rows, N = 32 ... 2^20", "hbm_peak_gbs": peak, "rows": rows}))
+    print(json.dumps({"landscape": "forward rows, N = 8 ... 2^20", "hbm_peak_gbs": peak, "rows": rows}))
     return 0
 
 
@@ -794,7 +796,7 @@ def main():
                     help="run one workload only, e.g. rows:16384:8192:c64, cols:4096:4096:c64, sar:c64")
     ap.add_argument("--option", action="append", default=[],
                     help="with --case rows/cols: plan option KEY=VALUE (repeatable), e.g. cluster=4")
-    ap.add_argument("--landscape", action="store_true", help="throughput against N = 32 ... 2^20, cold 1 GiB and hot 32 MiB")
+    ap.add_argument("--landscape", action="store_true", help="throughput against N = 8 ... 2^20, cold 1 GiB and hot 32 MiB")
     ap.add_argument("--sweep", action="store_true", help="hot vs cold throughput against the batch footprint")
     args = ap.parse_args()
     if args.sweep:

@@ -125,10 +125,12 @@ int fft_plan_destroy(fft_plan_t plan);
  *                memory (2-D tiled bulk copies of this GPU's own memory, no multicast) and takes the
  *                finished one out while the current one is transformed; 0 forbids it; -1 restores the
  *                default rules.
- *   "staged"     (rows plans, n = 16384) 1 selects the persistent kernel whose next transform arrives
+ *   "staged"     (rows plans) n = 16384: 1 selects the persistent kernel whose next transform arrives
  *                in shared memory through untiled bulk copies while the current one is computed; 0
  *                forbids it; -1 restores the default (on for fp16 storage with at least two transforms
- *                per multiprocessor).
+ *                per multiprocessor). n <= 32 with dist == n: by default one thread per transform, the
+ *                128 transforms of a CTA copied through shared memory in contiguous 16-byte pieces; 0
+ *                selects the plain kernel (several threads per transform at n = 32, direct loads).
  *   "prefetch"   d makes each CTA of a rows plan ask L2 for the input of the transform d tiles ahead
  *                (0 = off, -1 = the default: one wave ahead for n = 16384).
  *   "via_transpose"  1 makes a columns plan work the way the paper's four-pass pipeline does (Section
