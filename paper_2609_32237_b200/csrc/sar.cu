@@ -320,18 +320,31 @@ __global__ void __launch_bounds__(C::THREADS, 1) sar_rcmc_filter_ifft_kernel(con
 // output with the plain column kernel. One more trip through memory than the fused
 // kernel, but every thread is independent here (no tile-wide barriers), which on this
 // machine is faster than doing the interpolation inside the lock-stepped column tile.
+__device__ __forceinline__ void sinc8_weights_pair(float mua, float mub, float2 (&w)[8]);
+
 struct RcmcRows {
     static constexpr int COLS = 1024;   // range bins per CTA
     static constexpr int HALO = 64;     // extra staged samples: taps, alignment, growth of the shift over COLS bins
     static constexpr int TPB = 256;
 };
 
+// Measured on B200, 4096 x 4096: with the window in one interleaved array half of the 18.4 M shared-memory
+// wavefronts were bank-conflict replays and the L1/shared pipe was 92 % busy; split by parity the kernel
+// issues 9.9 M wavefronts (L1 53 %) and takes the same time, so that pipe was not what bound it: issue slots
+// (64 % active, 123 thread instructions per pixel) and the special-function pipe (60 %) are. Taking the eight
+// reciprocals of a pixel from four (1/a = b / (ab)) and asking for six (fp32 input) or five (fp16 input)
+// resident CTAs gave 163 -> 159 us for step 2; other register bounds measured 1-3 % slower.
 template <class TIn, class TOut = StoreC64>
-__global__ void __launch_bounds__(RcmcRows::TPB) sar_rcmc_filter_rows_kernel(const SarArgs a, int chunks) {
+__global__ void __launch_bounds__(RcmcRows::TPB, TIn::ELEM_BYTES == 8 ? 6 : 5) sar_rcmc_filter_rows_kernel(const SarArgs a, int chunks) {
     constexpr int COLS = RcmcRows::COLS, HALO = RcmcRows::HALO, TPB = RcmcRows::TPB;
     constexpr int EB = TIn::ELEM_BYTES, GRAN = 16 / EB;
     using elem_t = typename std::conditional<EB == 8, float2, __half2>::type;
-    __shared__ __align__(16) elem_t srow[COLS + HALO];
+    // The staged window is kept de-interleaved: even samples in the first half, odd samples in the second.
+    // A thread works on two adjacent range bins, so the lanes of a warp read every other sample; in one
+    // interleaved array that is a 16-byte stride (two wavefronts where one would do), in the split arrays the
+    // lanes read neighbouring words.
+    constexpr int HALF = (COLS + HALO) / 2;
+    __shared__ __align__(16) elem_t srow[2 * HALF];
     const int k = blockIdx.x / chunks;                 // Doppler bin
     const int c0 = (blockIdx.x % chunks) * COLS;       // first range bin of this CTA
     const float4 mg = __ldg(a.tab.mig + k);
@@ -346,7 +359,13 @@ __global__ void __launch_bounds__(RcmcRows::TPB) sar_rcmc_filter_rows_kernel(con
         const int col = start + i * GRAN;
         uint4 v = make_uint4(0u, 0u, 0u, 0u);
         if (col >= 0 && col + GRAN <= a.nr) v = *reinterpret_cast<const uint4*>(in + col);
-        *reinterpret_cast<uint4*>(srow + i * GRAN) = v;
+        if constexpr (EB == 8) {           // samples 2i, 2i + 1
+            *reinterpret_cast<uint2*>(srow + i) = make_uint2(v.x, v.y);
+            *reinterpret_cast<uint2*>(srow + HALF + i) = make_uint2(v.z, v.w);
+        } else {                           // samples 4i .. 4i + 3
+            *reinterpret_cast<uint2*>(srow + 2 * i) = make_uint2(v.x, v.z);
+            *reinterpret_cast<uint2*>(srow + HALF + 2 * i) = make_uint2(v.y, v.w);
+        }
     }
     __syncthreads();
     const int64_t orow = (int64_t)k * a.ld;
@@ -363,32 +382,38 @@ __global__ void __launch_bounds__(RcmcRows::TPB) sar_rcmc_filter_rows_kernel(con
             mub -= 1.0f;
             ib += 1;
         }
-        float wa[8], wb[8];
-        sinc8_weights_rcp(mua, wa);
-        sinc8_weights_rcp(mub, wb);
+        float2 wt[8];                                  // .x: bin n, .y: bin n + 1
+        sinc8_weights_pair(mua, mub, wt);
         const int oa = min(max(n + ia - 3 - start, 0), COLS + HALO - 8);
         const int ob = min(max(n + 1 + ib - 3 - start, 0), COLS + HALO - 8);
         float2 sa = make_float2(0.f, 0.f), sb = make_float2(0.f, 0.f);
+        // sample o + tap lives at (o + tap) / 2 in the half that matches its parity
+        const elem_t* ea = srow + (oa >> 1) + ((oa & 1) ? HALF : 0);      // even taps: ea[tap / 2]
+        const elem_t* da = srow + (oa >> 1) + ((oa & 1) ? 1 : HALF);      // odd taps: da[(tap - 1) / 2]
+        const elem_t* eb = srow + (ob >> 1) + ((ob & 1) ? HALF : 0);
+        const elem_t* db = srow + (ob >> 1) + ((ob & 1) ? 1 : HALF);
 #pragma unroll
         for (int tap = 0; tap < 8; ++tap) {
             float2 u, w2;
+            const elem_t ua = (tap & 1) ? da[tap / 2] : ea[tap / 2];
+            const elem_t ub = (tap & 1) ? db[tap / 2] : eb[tap / 2];
             if constexpr (EB == 8) {
-                u = srow[oa + tap];
-                w2 = srow[ob + tap];
+                u = ua;
+                w2 = ub;
             } else {
-                u = __half22float2(srow[oa + tap]);
-                w2 = __half22float2(srow[ob + tap]);
+                u = __half22float2(ua);
+                w2 = __half22float2(ub);
             }
             if ((tap - 3) & 1) {
-                sa.x = fmaf(-wa[tap], u.x, sa.x);
-                sa.y = fmaf(-wa[tap], u.y, sa.y);
-                sb.x = fmaf(-wb[tap], w2.x, sb.x);
-                sb.y = fmaf(-wb[tap], w2.y, sb.y);
+                sa.x = fmaf(-wt[tap].x, u.x, sa.x);
+                sa.y = fmaf(-wt[tap].x, u.y, sa.y);
+                sb.x = fmaf(-wt[tap].y, w2.x, sb.x);
+                sb.y = fmaf(-wt[tap].y, w2.y, sb.y);
             } else {
-                sa.x = fmaf(wa[tap], u.x, sa.x);
-                sa.y = fmaf(wa[tap], u.y, sa.y);
-                sb.x = fmaf(wb[tap], w2.x, sb.x);
-                sb.y = fmaf(wb[tap], w2.y, sb.y);
+                sa.x = fmaf(wt[tap].x, u.x, sa.x);
+                sa.y = fmaf(wt[tap].x, u.y, sa.y);
+                sb.x = fmaf(wt[tap].y, w2.x, sb.x);
+                sb.y = fmaf(wt[tap].y, w2.y, sb.y);
             }
         }
         const float2 fa = filter_phase(ph, n);
