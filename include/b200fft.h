@@ -37,6 +37,7 @@ enum {
 
 typedef struct b200fft_plan_s *fft_plan_t;
 typedef struct b200fft_sar_s *sar_rda_params_t;
+typedef struct b200fft_sar_shard_s *sar_rda_shard_t;
 
 /* ------------------------------------------------------------------------
  * Batched 1-D complex-to-complex transform (paper, Section "The M6 Memory
@@ -286,6 +287,59 @@ int sar_rda_form_image_host(const void *host_raw, sar_rda_params_t params, void 
 int sar_rda_run_step(const void *raw, sar_rda_params_t params, void *out, int step, void *stream);
 
 int sar_rda_params_destroy(sar_rda_params_t params);
+
+/* ------------------------------------------------------------------------
+ * Image formation split over `world` devices, one process per device (not in
+ * the paper, whose chain runs on one device; the decomposition follows from the
+ * chain's structure in Section "End to End: Range-Doppler SAR": range
+ * compression works on whole pulses, every later step on whole range-bin
+ * columns, and the interpolator of step 2 reaches a bounded number of bins
+ * along range). Rank r
+ *   1. range-compresses pulses [first_pulse, first_pulse + pulses) and stores
+ *      every compressed sample straight into the strip buffer of the rank that
+ *      owns its range bin (its own memory or a peer's, through the addresses the
+ *      caller passes in `strips`), and a second time into the neighbouring strip
+ *      whose halo it falls into: the exchange is part of the kernel's epilogue,
+ *      plain stores, no separate transpose or collective;
+ *   2. after every rank has finished step 1 (the caller synchronises: a barrier
+ *      of its process group after a stream synchronise), runs the azimuth FFT,
+ *      RCMC + filter and the inverse azimuth FFT on its strip and writes range
+ *      bins [first_bin, first_bin + bins) of the image, n_azimuth rows of `bins`
+ *      complex64 values.
+ * A strip buffer is n_azimuth rows of strip_width = halo_left + bins +
+ * halo_right elements of the intermediate type: the strip's bins and, on both
+ * sides, the neighbouring bins the interpolator reads (halo_right covers the
+ * largest range migration of the frame plus the taps); halo bins outside the
+ * frame are written as zeros by the rank that owns the pulse. The strip buffer
+ * is the first strip_bytes of the rank's workspace (workspace_bytes in all).
+ * world is 1, 2, 4 or 8; n_azimuth must be a multiple of world and n_range of
+ * 8 * world; halo_left + halo_right must not exceed bins (else
+ * B200FFT_ERR_UNSUPPORTED). Results equal the single-device chain to rounding
+ * (the per-bin coefficients are built in float64 for the strip's own origin).
+ * ---------------------------------------------------------------------- */
+typedef struct {
+    int64_t first_pulse, pulses;     /* rows of the raw frame this rank range-compresses */
+    int64_t first_bin, bins;         /* range bins of the image this rank forms */
+    int64_t halo_left, halo_right;   /* neighbouring bins kept on each side of the strip */
+    int64_t strip_width;             /* halo_left + bins + halo_right: row pitch of the strip buffer, in elements */
+    int64_t strip_bytes;             /* n_azimuth * strip_width elements of the intermediate type */
+    int64_t workspace_bytes;         /* the strip buffer followed by the second intermediate image */
+} sar_rda_shard_geometry;
+
+/* Host arithmetic only (no device needed): the geometry of rank `rank` of `world`. */
+int sar_rda_shard_geometry_of(const sar_rda_desc *scene, int32_t rank, int32_t world, sar_rda_shard_geometry *geometry);
+/* Tables and kernels for this rank on the current device. `scene` describes the whole frame. */
+int sar_rda_shard_create(sar_rda_shard_t *shard, const sar_rda_desc *scene, int32_t rank, int32_t world);
+int sar_rda_shard_get_geometry(sar_rda_shard_t shard, sar_rda_shard_geometry *geometry);
+/* This rank's workspace (device memory, 16-byte aligned, at least workspace_bytes, caller-owned). Its start is
+ * the strip buffer that every rank's step 1 stores into, so it must be memory the other ranks can address. */
+int sar_rda_shard_set_workspace(sar_rda_shard_t shard, void *device_ptr, size_t bytes);
+/* Step 1. raw_rows: this rank's pulses, `pulses` rows of n_range complex64 (device). strips: `world` device
+ * addresses (host array), strips[g] = the workspace of rank g as this process addresses it. Asynchronous. */
+int sar_rda_shard_range_compress(sar_rda_shard_t shard, const void *raw_rows, void *const *strips, void *stream);
+/* Step 2, after all ranks completed step 1. image_strip: n_azimuth x bins complex64 (device), not the workspace. */
+int sar_rda_shard_azimuth(sar_rda_shard_t shard, void *image_strip, void *stream);
+int sar_rda_shard_destroy(sar_rda_shard_t shard);
 
 #ifdef __cplusplus
 }

@@ -25,7 +25,8 @@ EXPORTS = [
     "b200fft_launch_count", "sar_rda_params_create", "sar_rda_workspace_bytes",
     "sar_rda_set_workspace", "sar_rda_form_image", "sar_rda_form_image_host", "sar_rda_run_step",
     "sar_rda_params_destroy", "fft_execute_noalloc", "sar_rda_set_option", "b200fft_tma_timeouts",
-    "fft_execute_bfp",
+    "fft_execute_bfp", "sar_rda_shard_geometry_of", "sar_rda_shard_create", "sar_rda_shard_get_geometry",
+    "sar_rda_shard_set_workspace", "sar_rda_shard_range_compress", "sar_rda_shard_azimuth", "sar_rda_shard_destroy",
 ]
 
 
@@ -72,7 +73,21 @@ def _load():
     L.fft_execute_noalloc.argtypes = [i64, i64, ci, vp, vp, vp]
     L.fft_execute_bfp.argtypes = [vp, vp, vp, vp, vp, vp]
     L.sar_rda_set_option.argtypes = [vp, ctypes.c_char_p, i64]
+    L.sar_rda_shard_geometry_of.argtypes = [ctypes.POINTER(SarRdaDesc), ctypes.c_int32, ctypes.c_int32,
+                                            ctypes.POINTER(SarShardGeometry)]
+    L.sar_rda_shard_create.argtypes = [ctypes.POINTER(vp), ctypes.POINTER(SarRdaDesc), ctypes.c_int32, ctypes.c_int32]
+    L.sar_rda_shard_get_geometry.argtypes = [vp, ctypes.POINTER(SarShardGeometry)]
+    L.sar_rda_shard_set_workspace.argtypes = [vp, vp, ctypes.c_size_t]
+    L.sar_rda_shard_range_compress.argtypes = [vp, vp, ctypes.POINTER(vp), vp]
+    L.sar_rda_shard_azimuth.argtypes = [vp, vp, vp]
+    L.sar_rda_shard_destroy.argtypes = [vp]
     return L
+
+
+class SarShardGeometry(ctypes.Structure):
+    _fields_ = [(name, ctypes.c_int64) for name in (
+        "first_pulse", "pulses", "first_bin", "bins", "halo_left", "halo_right", "strip_width", "strip_bytes",
+        "workspace_bytes")]
 
 
 _lib = _load()
@@ -183,6 +198,41 @@ def sar_rda_run_step(raw_ptr, params, out_ptr, step, stream=0):
 
 def sar_rda_params_destroy(params):
     _check(_lib.sar_rda_params_destroy(params), "sar_rda_params_destroy")
+
+
+def sar_rda_shard_geometry_of(desc: SarRdaDesc, rank: int, world: int) -> SarShardGeometry:
+    g = SarShardGeometry()
+    _check(_lib.sar_rda_shard_geometry_of(ctypes.byref(desc), rank, world, ctypes.byref(g)), "sar_rda_shard_geometry_of")
+    return g
+
+
+def sar_rda_shard_create(desc: SarRdaDesc, rank: int, world: int) -> int:
+    h = ctypes.c_void_p()
+    _check(_lib.sar_rda_shard_create(ctypes.byref(h), ctypes.byref(desc), rank, world), "sar_rda_shard_create")
+    return h.value
+
+
+def sar_rda_shard_get_geometry(shard) -> SarShardGeometry:
+    g = SarShardGeometry()
+    _check(_lib.sar_rda_shard_get_geometry(shard, ctypes.byref(g)), "sar_rda_shard_get_geometry")
+    return g
+
+
+def sar_rda_shard_set_workspace(shard, device_ptr, nbytes):
+    _check(_lib.sar_rda_shard_set_workspace(shard, device_ptr, nbytes), "sar_rda_shard_set_workspace")
+
+
+def sar_rda_shard_range_compress(shard, raw_rows_ptr, strip_ptrs, stream=0):
+    arr = (ctypes.c_void_p * len(strip_ptrs))(*strip_ptrs)
+    _check(_lib.sar_rda_shard_range_compress(shard, raw_rows_ptr, arr, stream), "sar_rda_shard_range_compress")
+
+
+def sar_rda_shard_azimuth(shard, image_strip_ptr, stream=0):
+    _check(_lib.sar_rda_shard_azimuth(shard, image_strip_ptr, stream), "sar_rda_shard_azimuth")
+
+
+def sar_rda_shard_destroy(shard):
+    _check(_lib.sar_rda_shard_destroy(shard), "sar_rda_shard_destroy")
 
 
 def sar_desc_from_scene(scene, intermediate_dtype=C64) -> SarRdaDesc:

@@ -807,6 +807,11 @@ struct Engine {
     template <class ST, bool CONJ, class Index>
     __device__ __forceinline__ void first_stage_dit_and_store_at(const float2* __restrict__ tw, void* out, float scale,
                                                                  Index&& index) {
+        first_stage_dit_emit<CONJ>(tw, scale, [&](int p, int q, float2 pa, float2 pb) { ST::store2(out, index(p, q), pa, pb); });
+    }
+    // The same, handing every finished pair (position p, column q, the two values) to the caller's `emit`.
+    template <bool CONJ, class Emit>
+    __device__ __forceinline__ void first_stage_dit_emit(const float2* __restrict__ tw, float scale, Emit&& emit) {
         using G = Geo<C, 1>;
         constexpr int V = G::V;
         static_assert(V >= 2, "register pairs");
@@ -816,7 +821,7 @@ struct Engine {
             const int q = c % W, lo = c / W;
             pa = make_float2(pa.x * scale, (CONJ ? -pa.y : pa.y) * scale);
             pb = make_float2(pb.x * scale, (CONJ ? -pb.y : pb.y) * scale);
-            ST::store2(out, index(k * G::Ls + lo, q), pa, pb);
+            emit(k * G::Ls + lo, q, pa, pb);
         });
     }
 

@@ -8,13 +8,12 @@
 //           output scaled by 1/n_azimuth (the paper's fixed-shift schedule)
 //   step 2  fused range cell migration correction (8-tap sinc), azimuth filter
 //           exp(+j 4 pi R0 (D - 1) / lambda) and inverse azimuth FFT on column tiles
-// Between the steps the image lives in the caller's workspace. Its layout is the library's own
-// choice, and by default it is the slab layout of fft_core.cuh with 32-byte granules (4 complex64
-// or 8 complex-half range bins): every column tile of the azimuth transforms is then row segments
-// inside one contiguous slab instead of 32-byte pieces at a pitch of a whole image row, range
-// compression still writes whole sectors, and step 2 runs as a row-wise pass over slabs (RCMC +
-// filter, slab to slab) followed by the inverse column transform that writes the row-major image.
-// The row-major intermediate of the first design stays selectable (option "layout" = 0).
+// Between the steps the image lives in the caller's workspace, row-major by default (the azimuth transforms
+// read it as column tiles in place; step 2 runs as a row pass, RCMC + filter, followed by the inverse column
+// transform). Two other organisations are selectable (option "layout"): the slab layout of fft_core.cuh with
+// 32-byte granules, and azimuth transforms by transposition (the paper's four-pass form).
+// The azimuth steps also run on a strip of range bins cut from a larger image (sar_rda_shard_*): the strip is
+// then a frame of its own whose first range bin sits `first_bin` bins into the whole swath.
 // The filter and the migration are affine in the range index with per-Doppler-bin
 // coefficients, built once in float64. The paper's four numerical fixes are kept:
 // baseband filter (D - 1); phase in cycles with a split that makes the fp32
@@ -48,11 +47,26 @@ struct SarArgs {
     int nr;
     float scale;
     int na;              // rows of the image (n_azimuth)
+    // Row pass of step 2: output column j (0 .. out_cols - 1) is range bin j + col0 of the input frame and is
+    // stored at a row pitch of out_ld elements. Whole image: col0 = 0, out_cols = nr, out_ld = ld.
+    int col0, out_cols;
+    int64_t out_ld;
+    // Range compression that scatters its rows over the strips of a column-strip decomposition: strip g covers
+    // range bins [g * strip_cols - halo_l, (g + 1) * strip_cols + halo_r) of the whole frame, stored as
+    // n_azimuth rows of sw = halo_l + strip_cols + halo_r elements at strip[g] (an address this device can
+    // store to: its own memory or a peer's). Bins outside the frame are written as zeros.
+    struct {
+        unsigned long long strip[8];
+        int world, strip_cols, halo_l, halo_r, sw;
+        int64_t row0;    // first pulse of this launch within the whole frame
+    } sh;
 };
 
 // ---------------------------------------------------------------- step 0
-// SLAB: the output goes to the slab layout (granules of 32 bytes) instead of row-major.
-template <class C, class TOut, bool SLAB>
+// MODE 0: row-major output; 1: the slab layout (granules of 32 bytes); 2: scattered over the strips of a
+// column-strip decomposition (SarArgs::sh), every pair stored to the strip that owns it and to the neighbour
+// whose halo it falls into.
+template <class C, class TOut, int MODE>
 __global__ void __launch_bounds__(C::THREADS, C::MINB) sar_range_compress_kernel(const SarArgs a) {
     extern __shared__ __align__(16) float2 smem_dyn[];
     static_assert(C::W == 1, "range compression works on contiguous rows");
@@ -88,12 +102,25 @@ __global__ void __launch_bounds__(C::THREADS, C::MINB) sar_range_compress_kernel
     }
     e.template dit<false>(sm, a.tw);
     if (!active) return;
-    if constexpr (SLAB) {
+    if constexpr (MODE == 1) {
         constexpr int GS = 32 / TOut::ELEM_BYTES;
         const int64_t na = a.na;
         e.template first_stage_dit_and_store_at<TOut, true>(a.tw, a.out, 1.0f, [&](int p, int) -> int64_t {
             return ((int64_t)(p / GS) * na + tile) * GS + (p % GS);
         });
+    } else if constexpr (MODE == 2) {
+        const int sc = a.sh.strip_cols, hl = a.sh.halo_l, hr = a.sh.halo_r, last = a.sh.world - 1;
+        const int64_t rowoff = (a.sh.row0 + tile) * (int64_t)a.sh.sw;      // this pulse's row in every strip
+        auto strip = [&](int g) { return reinterpret_cast<void*>(a.sh.strip[g]); };
+        e.template first_stage_dit_emit<true>(a.tw, 1.0f, [&](int p, int, float2 pa, float2 pb) {
+            const int g = p / sc, lc = p - g * sc;                       // sc, hl, hr are even: a pair stays together
+            TOut::store2(strip(g), rowoff + hl + lc, pa, pb);
+            if (lc < hr && g > 0) TOut::store2(strip(g - 1), rowoff + hl + sc + lc, pa, pb);
+            if (lc >= sc - hl && g < last) TOut::store2(strip(g + 1), rowoff + lc - (sc - hl), pa, pb);
+        });
+        const float2 z = make_float2(0.f, 0.f);
+        for (int i = 2 * t; i < hl; i += 2 * C::T) TOut::store2(strip(0), rowoff + i, z, z);
+        for (int i = 2 * t; i < hr; i += 2 * C::T) TOut::store2(strip(last), rowoff + hl + sc + i, z, z);
     } else {
         e.template first_stage_dit_and_store<TOut, true>(a.tw, a.out, base, a.ld, 1.0f);
     }
@@ -346,7 +373,8 @@ __global__ void __launch_bounds__(RcmcRows::TPB, TIn::ELEM_BYTES == 8 ? 6 : 5) s
     constexpr int HALF = (COLS + HALO) / 2;
     __shared__ __align__(16) elem_t srow[2 * HALF];
     const int k = blockIdx.x / chunks;                 // Doppler bin
-    const int c0 = (blockIdx.x % chunks) * COLS;       // first range bin of this CTA
+    const int j0 = (blockIdx.x % chunks) * COLS;       // first output column of this CTA
+    const int c0 = j0 + a.col0;                        // its range bin in the input frame
     const float4 mg = __ldg(a.tab.mig + k);
     const float4 ph = __ldg(a.tab.phs + k);
     const float2 step = __ldg(a.tab.stp + k);
@@ -368,11 +396,12 @@ __global__ void __launch_bounds__(RcmcRows::TPB, TIn::ELEM_BYTES == 8 ? 6 : 5) s
         }
     }
     __syncthreads();
-    const int64_t orow = (int64_t)k * a.ld;
+    const int64_t orow = (int64_t)k * a.out_ld;
     const float g = mg.x + mg.y;
 #pragma unroll
     for (int h = 0; h < COLS / (2 * TPB); ++h) {
-        const int n = c0 + h * 2 * TPB + 2 * threadIdx.x;          // range bins n, n + 1
+        const int j = j0 + h * 2 * TPB + 2 * threadIdx.x;          // output columns j, j + 1
+        const int n = j + a.col0;                                  // range bins n, n + 1
         int ia, ib;
         float mua, mub;
         migration(mg, n, ia, mua);
@@ -419,7 +448,7 @@ __global__ void __launch_bounds__(RcmcRows::TPB, TIn::ELEM_BYTES == 8 ? 6 : 5) s
         const float2 fa = filter_phase(ph, n);
         const float2 fb = cmul(fa, step);
         const float2 ya = cmul(sa, fa), yb = cmul(sb, fb);
-        TOut::store2(a.out, orow + n, ya, yb);
+        if (j < a.out_cols) TOut::store2(a.out, orow + j, ya, yb);
     }
 }
 
@@ -611,8 +640,10 @@ __device__ double round_to_bits(double v, int bits) {
     return ldexp(rint(ldexp(m, bits)), ex - bits);
 }
 
+// nr: range bins of the whole frame, whose centre bin nr / 2 is at r_center; first_bin: range bin of the whole
+// frame that the tables call n = 0 (0 for the whole frame, a strip's first bin otherwise).
 __global__ void sar_build_doppler_tables(float4* mig, float4* phs, float2* stp, int na, int nr, double wavelength,
-                                         double prf, double velocity, double r_center, double dr) {
+                                         double prf, double velocity, double r_center, double dr, double first_bin) {
     const int k = blockIdx.x * blockDim.x + threadIdx.x;
     if (k >= na) return;
     const int kk = (k < na / 2) ? k : k - na;
@@ -624,12 +655,12 @@ __global__ void sar_build_doppler_tables(float4* mig, float4* phs, float2* stp, 
     const double d_minus_1 = -u / (1.0 + sq);              // D - 1
     // migration in bins: dn(n) = (r_center/dr - nr/2 + n) * (1/D - 1) = a0 + n g
     const double gslope = inv_d_minus_1;
-    const double a0 = (r_center / dr - (double)(nr / 2)) * gslope;
+    const double a0 = (r_center / dr - (double)(nr / 2) + first_bin) * gslope;
     const double g_hi = round_to_bits(gslope, 10);
     const double a_int = floor(a0);
     mig[k] = make_float4((float)g_hi, (float)(gslope - g_hi), (float)(a0 - a_int), __int_as_float((int)a_int));
     // filter phase in cycles: (2/lambda) R0(n) (D - 1) = A + n B
-    const double A = (2.0 / wavelength) * (r_center - (double)(nr / 2) * dr) * d_minus_1;
+    const double A = (2.0 / wavelength) * (r_center + (first_bin - (double)(nr / 2)) * dr) * d_minus_1;
     const double B = (2.0 * dr / wavelength) * d_minus_1;
     const double b_hi = round_to_bits(B, 10);
     phs[k] = make_float4((float)(A - floor(A)), (float)b_hi, (float)(B - b_hi), 0.0f);
@@ -639,12 +670,12 @@ __global__ void sar_build_doppler_tables(float4* mig, float4* phs, float2* stp, 
 }
 
 // ---------------------------------------------------------------- host side
-template <class C, class TOut, bool SLAB>
+template <class C, class TOut, int MODE>
 cudaError_t launch_range(const SarArgs& a, cudaStream_t st) {
     static bool done[64] = {};
-    cudaError_t e = ensure_smem(sar_range_compress_kernel<C, TOut, SLAB>, C::SMEM_BYTES, done);
+    cudaError_t e = ensure_smem(sar_range_compress_kernel<C, TOut, MODE>, C::SMEM_BYTES, done);
     if (e != cudaSuccess) return e;
-    return launch_tiles<C>(sar_range_compress_kernel<C, TOut, SLAB>, a, a.tiles, st);
+    return launch_tiles<C>(sar_range_compress_kernel<C, TOut, MODE>, a, a.tiles, st);
 }
 template <class C, class TIn, bool SLAB>
 cudaError_t launch_rcmc(const SarArgs& a, cudaStream_t st) {
@@ -668,27 +699,29 @@ cudaError_t launch_rcmc_pass(const SarArgs& a, cudaStream_t st) {
 
 struct SarEntry {
     int n, dtype, w, tw_total;
-    bool slab;
+    int mode;            // 0 row-major, 1 slab layout, 2 (range compression only) scattered over column strips
     cudaError_t (*launch)(const SarArgs&, cudaStream_t);
     cudaError_t (*build_tw)(float2*, cudaStream_t);
 };
-template <class C, class T, bool RANGE, bool SLAB>
+template <class C, class T, bool RANGE, int MODE>
 constexpr SarEntry sar_entry() {
     if constexpr (RANGE)
-        return SarEntry{C::N, T::ELEM_BYTES == 8 ? 0 : 1, C::W, C::TW_TOTAL, SLAB, &launch_range<C, T, SLAB>, &launch_build_tw<C>};
+        return SarEntry{C::N, T::ELEM_BYTES == 8 ? 0 : 1, C::W, C::TW_TOTAL, MODE, &launch_range<C, T, MODE>, &launch_build_tw<C>};
     else
-        return SarEntry{C::N, T::ELEM_BYTES == 8 ? 0 : 1, C::W, C::TW_TOTAL, SLAB, &launch_rcmc<C, T, SLAB>, &launch_build_tw<C>};
+        return SarEntry{C::N, T::ELEM_BYTES == 8 ? 0 : 1, C::W, C::TW_TOTAL, MODE, &launch_rcmc<C, T, MODE == 1>, &launch_build_tw<C>};
 }
-#define SAR_QUAD(C, RANGE)                                                                        \
-    sar_entry<C, StoreC64, RANGE, false>(), sar_entry<C, StoreC32H, RANGE, false>(),             \
-    sar_entry<C, StoreC64, RANGE, true>(), sar_entry<C, StoreC32H, RANGE, true>()
-static const SarEntry k_range[] = {SAR_QUAD(R1024p, true), SAR_QUAD(R2048, true), SAR_QUAD(R4096, true), SAR_QUAD(R8192, true)};
+#define SAR_QUAD(C, RANGE)                                                                \
+    sar_entry<C, StoreC64, RANGE, 0>(), sar_entry<C, StoreC32H, RANGE, 0>(),             \
+    sar_entry<C, StoreC64, RANGE, 1>(), sar_entry<C, StoreC32H, RANGE, 1>()
+#define SAR_SHARD(C) sar_entry<C, StoreC64, true, 2>(), sar_entry<C, StoreC32H, true, 2>()
+static const SarEntry k_range[] = {SAR_QUAD(R1024p, true), SAR_QUAD(R2048, true), SAR_QUAD(R4096, true), SAR_QUAD(R8192, true),
+                                   SAR_SHARD(R1024p),      SAR_SHARD(R2048),      SAR_SHARD(R4096),      SAR_SHARD(R8192)};
 static const SarEntry k_rcmc[] = {SAR_QUAD(T1024, false), SAR_QUAD(T2048, false), SAR_QUAD(T4096, false)};
 
 template <size_t K>
-static const SarEntry* find(const SarEntry (&tab)[K], int n, int dtype, bool slab) {
+static const SarEntry* find(const SarEntry (&tab)[K], int n, int dtype, int mode) {
     for (const SarEntry& e : tab)
-        if (e.n == n && e.dtype == dtype && e.slab == slab) return &e;
+        if (e.n == n && e.dtype == dtype && e.mode == mode) return &e;
     return nullptr;
 }
 
@@ -745,6 +778,19 @@ struct b200fft_sar_s {
     float2* stp;
     void* workspace;
     size_t workspace_bytes;
+    // A strip of range bins cut from a larger frame (sar_rda_shard_*): steps 1 and 2 only. The frame described
+    // by `d` is the strip with its halos; step 2 keeps out_cols columns starting at column col0.
+    bool strip;
+    int col0;
+    int64_t out_cols;
+};
+
+// how a strip sits in the whole frame
+struct SarStrip {
+    int64_t nr_whole;    // range bins of the whole frame
+    int64_t first_bin;   // range bin of the whole frame at which column 0 of the strip's frame sits (may be negative)
+    int col0;            // first kept column
+    int64_t out_cols;    // kept columns
 };
 
 static void sar_release(b200fft_sar_s* p) {
@@ -761,7 +807,13 @@ static size_t image_bytes(const b200fft_sar_s* p) {
     return (size_t)p->d.n_azimuth * (size_t)p->d.n_range * (p->d.intermediate_dtype == B200FFT_C64 ? 8 : 4);
 }
 
-extern "C" int sar_rda_params_create(sar_rda_params_t* params, const sar_rda_desc* d) {
+static int sar_create(sar_rda_params_t* params, const sar_rda_desc* d, const SarStrip* strip);
+
+extern "C" int sar_rda_params_create(sar_rda_params_t* params, const sar_rda_desc* d) { return sar_create(params, d, nullptr); }
+
+// strip == nullptr: the whole chain on the frame `d`. Otherwise `d` describes the strip's own frame (n_range =
+// its columns with halos; r_center_m still that of the whole frame) and only the azimuth steps are prepared.
+static int sar_create(sar_rda_params_t* params, const sar_rda_desc* d, const SarStrip* strip) {
     if (!params || !d) return B200FFT_ERR_INVALID_ARG;
     *params = nullptr;
     if (d->n_azimuth <= 0 || d->n_range <= 0 || d->carrier_hz <= 0 || d->bandwidth_hz <= 0 || d->fs_hz <= 0 ||
@@ -776,14 +828,18 @@ extern "C" int sar_rda_params_create(sar_rda_params_t* params, const sar_rda_des
         if (4.0 * u / ((1.0 + sq) * sq) >= 1.0) return B200FFT_ERR_UNSUPPORTED;
     }
     const long long pulse_samples = llround(d->pulse_s * d->fs_hz);
-    if (pulse_samples < 1 || pulse_samples > d->n_range) return B200FFT_ERR_INVALID_ARG;
+    if (!strip && (pulse_samples < 1 || pulse_samples > d->n_range)) return B200FFT_ERR_INVALID_ARG;
 
     b200fft_sar_s* p = new (std::nothrow) b200fft_sar_s();
     if (!p) return B200FFT_ERR_ALLOC;
     p->d = *d;
     const int na = (int)d->n_azimuth, nr = (int)d->n_range, dt = d->intermediate_dtype;
-    p->range = find(k_range, nr, dt, false);
-    p->range_slab = find(k_range, nr, dt, true);
+    p->strip = strip != nullptr;
+    p->col0 = strip ? strip->col0 : 0;
+    p->out_cols = strip ? strip->out_cols : nr;
+    const int ocols = (int)p->out_cols;        // columns the inverse azimuth transform runs on
+    p->range = strip ? nullptr : find(k_range, nr, dt, 0);
+    p->range_slab = strip ? nullptr : find(k_range, nr, dt, 1);
     // Column tiles of the row-major layout: the persistent streaming kernel where it is compiled (4096 rows) and
     // the image gives every multiprocessor several tiles; else, with fp16 intermediates, the wider tile on a
     // cluster of two CTAs (32-byte instead of 16-byte row segments); else the plain 4-column tile.
@@ -792,25 +848,25 @@ extern "C" int sar_rda_params_create(sar_rda_params_t* params, const sar_rda_des
         int dev = 0;
         if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     }
-    auto cols_kernel = [&](bool inverse, int dtype) {
-        if (nr / 4 > sms) {
+    auto cols_kernel = [&](bool inverse, int dtype, int cols) {
+        if (cols / 4 > sms) {
             const KernelEntry* k = find_cols_kernel(na, inverse, dtype, dtype, 0, VAR_STREAM);
-            if (k && k->n >= 4096 && nr % k->w == 0) return k;
+            if (k && k->n >= 4096 && cols % k->w == 0) return k;
         }
         if (dtype == B200FFT_C32H) {
             const KernelEntry* k = find_cols_kernel(na, inverse, dtype, dtype, 0, VAR_WIDE_CLUSTER);
-            if (k && nr % k->w == 0) return k;
+            if (k && cols % k->w == 0) return k;
         }
         return find_cols_kernel(na, inverse, dtype, dtype, 1);
     };
-    p->azfft = cols_kernel(false, dt);
-    p->rcmc = find(k_rcmc, na, dt, false);
-    p->rcmc_slab = find(k_rcmc, na, dt, true);
-    p->azifft = cols_kernel(true, B200FFT_C64);
+    p->azfft = cols_kernel(false, dt, nr);
+    p->rcmc = find(k_rcmc, na, dt, 0);
+    p->rcmc_slab = find(k_rcmc, na, dt, 1);
+    p->azifft = cols_kernel(true, B200FFT_C64, ocols);
     p->azifft_h = nullptr;
-    if (dt == B200FFT_C32H && nr / 4 > sms) {
+    if (dt == B200FFT_C32H && ocols / 4 > sms && p->rcmc) {
         const KernelEntry* k = find_cols_kernel(na, true, B200FFT_C32H, B200FFT_C64, 0, VAR_STREAM);
-        if (k && nr % k->w == 0 && k->tw_total == p->rcmc->tw_total) p->azifft_h = k;
+        if (k && ocols % k->w == 0 && k->tw_total == p->rcmc->tw_total) p->azifft_h = k;
     }
     for (int i = 0; i < 2; ++i) {
         p->azfft_slab[i] = find_sar_cols_kernel(na, 2 << i, false, dt, dt);
@@ -822,18 +878,20 @@ extern "C" int sar_rda_params_create(sar_rda_params_t* params, const sar_rda_des
     {   // the row-major row pass stages COLS + HALO samples: the shift may grow by at most HALO - 16 bins over COLS bins
         const double aa = wavelength * d->prf_hz / (4.0 * d->velocity_mps), u = aa * aa, sq = sqrt(1.0 - u);
         const double gmax = u / ((1.0 + sq) * sq);
-        p->can_unfuse = p->azifft != nullptr && nr % RcmcRows::COLS == 0 &&
+        // (a strip's row pass may end inside a CTA's 1024 columns: the kernel checks the column before it stores)
+        p->can_unfuse = p->azifft != nullptr && (strip ? (ocols % p->azifft->w == 0 && ocols % 2 == 0) : nr % RcmcRows::COLS == 0) &&
                         gmax * RcmcRows::COLS + 16.0 <= (double)RcmcRows::HALO;
     }
-    p->can_slab = p->range_slab && p->rcmc_slab && p->azfft_slab[0] && p->azfft_slab[1] && p->azifft_slab[0] &&
+    p->can_slab = !strip && p->range_slab && p->rcmc_slab && p->azfft_slab[0] && p->azfft_slab[1] && p->azifft_slab[0] &&
                   p->azifft_slab[1] && row_pass_ok;
     p->rows_fwd = find_rows_kernel(na, false, dt, dt, 1, nr);
     p->rows_inv = find_rows_kernel(na, true, B200FFT_C64, B200FFT_C64, 1, nr);
-    p->can_transpose = p->rows_fwd && p->rows_inv && p->rows_fwd->tw_total == p->rows_inv->tw_total && p->can_unfuse;
+    p->can_transpose = !strip && p->rows_fwd && p->rows_inv && p->rows_fwd->tw_total == p->rows_inv->tw_total && p->can_unfuse;
     p->layout = 0;
     p->tile_columns = 4;
     p->fused = p->layout == 0 && !p->can_unfuse;
-    if (!p->range || !p->azfft || !p->rcmc || d->n_azimuth > 16384 || d->n_range > 16384 || nr % p->rcmc->w) {
+    if ((!strip && !p->range) || !p->azfft || !p->rcmc || d->n_azimuth > 16384 || d->n_range > 16384 || nr % p->rcmc->w ||
+        nr % p->azfft->w || (strip && p->fused)) {
         delete p;
         return B200FFT_ERR_UNSUPPORTED;
     }
@@ -846,9 +904,9 @@ extern "C" int sar_rda_params_create(sar_rda_params_t* params, const sar_rda_des
         delete p;                  // every azimuth kernel reads the one table built below
         return B200FFT_ERR_UNSUPPORTED;
     }
-    bool ok = cudaMalloc(&p->tw_range, sizeof(float2) * (size_t)p->range->tw_total) == cudaSuccess &&
+    bool ok = (strip || (cudaMalloc(&p->tw_range, sizeof(float2) * (size_t)p->range->tw_total) == cudaSuccess &&
+                         cudaMalloc(&p->H, sizeof(float2) * (size_t)nr) == cudaSuccess)) &&
               cudaMalloc(&p->tw_az, sizeof(float2) * (size_t)p->rcmc->tw_total) == cudaSuccess &&
-              cudaMalloc(&p->H, sizeof(float2) * (size_t)nr) == cudaSuccess &&
               cudaMalloc(&p->mig, sizeof(float4) * (size_t)na) == cudaSuccess &&
               cudaMalloc(&p->phs, sizeof(float4) * (size_t)na) == cudaSuccess &&
               cudaMalloc(&p->stp, sizeof(float2) * (size_t)na) == cudaSuccess;
@@ -860,14 +918,15 @@ extern "C" int sar_rda_params_create(sar_rda_params_t* params, const sar_rda_des
     }
     const double dr = kLight / (2.0 * d->fs_hz);
     const double kappa = (d->bandwidth_hz / d->pulse_s) / (d->fs_hz * d->fs_hz);
-    ok = p->range->build_tw(p->tw_range, 0) == cudaSuccess && p->rcmc->build_tw(p->tw_az, 0) == cudaSuccess;
+    ok = (strip || p->range->build_tw(p->tw_range, 0) == cudaSuccess) && p->rcmc->build_tw(p->tw_az, 0) == cudaSuccess;
     if (ok && p->can_transpose)
         ok = cudaMalloc(&p->tw_rows, sizeof(float2) * (size_t)p->rows_fwd->tw_total) == cudaSuccess &&
              p->rows_fwd->build_tw(p->tw_rows, 0) == cudaSuccess;
-    sar_build_matched_filter<<<(nr + 127) / 128, 128>>>(p->H, nr, (int)pulse_samples, kappa);
-    sar_build_doppler_tables<<<(na + 127) / 128, 128>>>(p->mig, p->phs, p->stp, na, nr, wavelength, d->prf_hz,
-                                                       d->velocity_mps, d->r_center_m, dr);
-    g_launch_count.fetch_add(2, std::memory_order_relaxed);
+    if (!strip) sar_build_matched_filter<<<(nr + 127) / 128, 128>>>(p->H, nr, (int)pulse_samples, kappa);
+    sar_build_doppler_tables<<<(na + 127) / 128, 128>>>(p->mig, p->phs, p->stp, na, strip ? (int)strip->nr_whole : nr, wavelength,
+                                                       d->prf_hz, d->velocity_mps, d->r_center_m, dr,
+                                                       strip ? (double)strip->first_bin : 0.0);
+    g_launch_count.fetch_add(strip ? 1 : 2, std::memory_order_relaxed);
     ok = ok && cudaGetLastError() == cudaSuccess && cudaStreamSynchronize(0) == cudaSuccess;
     if (!ok) {
         sar_release(p);
@@ -911,6 +970,7 @@ extern "C" int sar_rda_run_step(const void* raw, sar_rda_params_t p, void* out, 
         f.slab_stride = na * gcols;
         f.dist = gcols;
     };
+    if (p->strip && step == 0) return B200FFT_ERR_INVALID_ARG;     // a strip is filled by sar_rda_shard_range_compress
     if (step == 0) {
         if (!raw) return B200FFT_ERR_INVALID_ARG;
         if (reinterpret_cast<uintptr_t>(raw) % 16) return B200FFT_ERR_ALIGNMENT;
@@ -942,6 +1002,7 @@ extern "C" int sar_rda_run_step(const void* raw, sar_rda_params_t p, void* out, 
         a.in = buf0; a.out = out; a.tw = p->tw_az;
         a.tab = SarTables{p->H, p->mig, p->phs, p->stp};
         a.ld = nr; a.nr = (int)nr; a.na = (int)na; a.scale = 1.0f;
+        a.col0 = 0; a.out_cols = (int)nr; a.out_ld = nr;
         const int chunks = (int)(nr / RcmcRows::COLS);
         if (dt == B200FFT_C64)
             sar_rcmc_filter_rows_kernel<StoreC64><<<(unsigned)(na * chunks), RcmcRows::TPB, 0, st>>>(a, chunks);
@@ -989,7 +1050,9 @@ extern "C" int sar_rda_run_step(const void* raw, sar_rda_params_t p, void* out, 
         f.out_dist = nr;                    // the image leaves row-major
         return ok(k->launch(f, st));
     }
-    const int chunks = (int)(nr / RcmcRows::COLS);
+    const int64_t oc = p->out_cols;          // columns kept (all of them unless this is a strip with halos)
+    const int chunks = (int)((oc + RcmcRows::COLS - 1) / RcmcRows::COLS);
+    a.col0 = p->col0; a.out_cols = (int)oc; a.out_ld = oc;
     // With fp16 intermediates the row pass writes a second fp16 image (one more rounding, as in the paper's
     // four-pass accounting of 40 bytes per pixel) where the inverse column kernel for it is compiled; else the
     // complex64 output image, on which the inverse column pass then runs in place.
@@ -1006,12 +1069,13 @@ extern "C" int sar_rda_run_step(const void* raw, sar_rda_params_t p, void* out, 
     if (cudaGetLastError() != cudaSuccess) return B200FFT_ERR_CUDA;
     const KernelEntry* inv = half_image ? p->azifft_h : p->azifft;
     f.in = half_image ? buf1 : out; f.out = out;
-    f.tiles = nr / inv->w; f.dist = nr;
+    f.tiles = oc / inv->w; f.dist = oc;
     return ok(inv->launch(f, st));
 }
 
 extern "C" int sar_rda_set_option(sar_rda_params_t p, const char* key, int64_t value) {
     if (!p || !key) return B200FFT_ERR_INVALID_ARG;
+    if (p->strip) return B200FFT_ERR_UNSUPPORTED;
     if (std::strcmp(key, "fused_rcmc") == 0) {
         if (!value && p->layout == 0 && !p->can_unfuse) return B200FFT_ERR_UNSUPPORTED;
         if (value && p->layout == 2) return B200FFT_ERR_UNSUPPORTED;
@@ -1060,5 +1124,126 @@ extern "C" int sar_rda_params_destroy(sar_rda_params_t p) {
     if (!p) return B200FFT_ERR_INVALID_ARG;
     sar_release(p);
     delete p;
+    return B200FFT_OK;
+}
+
+// ---------------------------------------------------------------- column-strip decomposition over several devices
+struct b200fft_sar_shard_s {
+    b200fft_sar_s* whole;      // tables and kernel of the range compression (whole range lines)
+    b200fft_sar_s* strip;      // azimuth steps on this rank's strip
+    const SarEntry* scatter;   // range compression that stores into every rank's strip
+    sar_rda_shard_geometry g;
+    int rank, world;
+};
+
+extern "C" int sar_rda_shard_geometry_of(const sar_rda_desc* d, int32_t rank, int32_t world, sar_rda_shard_geometry* g) {
+    if (!d || !g) return B200FFT_ERR_INVALID_ARG;
+    if (world != 1 && world != 2 && world != 4 && world != 8) return B200FFT_ERR_INVALID_ARG;
+    if (rank < 0 || rank >= world) return B200FFT_ERR_INVALID_ARG;
+    if (d->n_azimuth <= 0 || d->n_range <= 0 || d->carrier_hz <= 0 || d->fs_hz <= 0 || d->prf_hz <= 0 || d->velocity_mps <= 0 ||
+        d->r_center_m <= 0)
+        return B200FFT_ERR_INVALID_ARG;
+    if (d->intermediate_dtype != B200FFT_C64 && d->intermediate_dtype != B200FFT_C32H) return B200FFT_ERR_INVALID_ARG;
+    if (d->n_azimuth % world || d->n_range % (8 * world)) return B200FFT_ERR_UNSUPPORTED;
+    const double wavelength = kLight / d->carrier_hz, dr = kLight / (2.0 * d->fs_hz);
+    const double aa = wavelength * d->prf_hz / (4.0 * d->velocity_mps);
+    if (aa >= 0.5) return B200FFT_ERR_INVALID_ARG;
+    const double u = aa * aa, sq = sqrt(1.0 - u);
+    // largest migration in the frame: far edge of the swath at the Doppler edge
+    const double far_bin = d->r_center_m / dr - (double)(d->n_range / 2) + (double)(d->n_range - 1);
+    const double smax = far_bin * (u / ((1.0 + sq) * sq));
+    if (smax < 0.0 || smax > 4096.0) return B200FFT_ERR_UNSUPPORTED;
+    const int64_t bins = d->n_range / world;
+    g->first_pulse = (int64_t)rank * (d->n_azimuth / world);
+    g->pulses = d->n_azimuth / world;
+    g->first_bin = (int64_t)rank * bins;
+    g->bins = bins;
+    g->halo_left = 8;                                               // taps reach 3 bins back; 8 keeps every row 32-byte aligned
+    g->halo_right = (((int64_t)ceil(smax) + 5) + 7) / 8 * 8;        // largest integer shift + 4 taps ahead
+    if (world > 1 && g->halo_left + g->halo_right > bins) return B200FFT_ERR_UNSUPPORTED;
+    g->strip_width = g->halo_left + bins + g->halo_right;
+    const int64_t eb = d->intermediate_dtype == B200FFT_C64 ? 8 : 4;
+    g->strip_bytes = d->n_azimuth * g->strip_width * eb;
+    g->workspace_bytes = 2 * g->strip_bytes;
+    return B200FFT_OK;
+}
+
+extern "C" int sar_rda_shard_create(sar_rda_shard_t* out, const sar_rda_desc* d, int32_t rank, int32_t world) {
+    if (!out || !d) return B200FFT_ERR_INVALID_ARG;
+    *out = nullptr;
+    sar_rda_shard_geometry g;
+    int rc = sar_rda_shard_geometry_of(d, rank, world, &g);
+    if (rc != B200FFT_OK) return rc;
+    b200fft_sar_shard_s* s = new (std::nothrow) b200fft_sar_shard_s();
+    if (!s) return B200FFT_ERR_ALLOC;
+    s->g = g;
+    s->rank = rank;
+    s->world = world;
+    s->scatter = find(k_range, (int)d->n_range, d->intermediate_dtype, 2);
+    rc = s->scatter ? sar_create(&s->whole, d, nullptr) : B200FFT_ERR_UNSUPPORTED;
+    if (rc == B200FFT_OK) {
+        sar_rda_desc sd = *d;
+        sd.n_range = g.strip_width;
+        const SarStrip geo{d->n_range, g.first_bin - g.halo_left, (int)g.halo_left, g.bins};
+        rc = sar_create(&s->strip, &sd, &geo);
+    }
+    if (rc != B200FFT_OK) {
+        if (s->whole) sar_rda_params_destroy(s->whole);
+        delete s;
+        return rc;
+    }
+    *out = s;
+    return B200FFT_OK;
+}
+
+extern "C" int sar_rda_shard_get_geometry(sar_rda_shard_t s, sar_rda_shard_geometry* g) {
+    if (!s || !g) return B200FFT_ERR_INVALID_ARG;
+    *g = s->g;
+    return B200FFT_OK;
+}
+
+extern "C" int sar_rda_shard_set_workspace(sar_rda_shard_t s, void* ptr, size_t bytes) {
+    if (!s || !ptr) return B200FFT_ERR_INVALID_ARG;
+    if (bytes < (size_t)s->g.workspace_bytes) return B200FFT_ERR_WORKSPACE;
+    return sar_rda_set_workspace(s->strip, ptr, bytes);
+}
+
+extern "C" int sar_rda_shard_range_compress(sar_rda_shard_t s, const void* raw_rows, void* const* strips, void* stream) {
+    if (!s || !raw_rows || !strips) return B200FFT_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(raw_rows) % 16) return B200FFT_ERR_ALIGNMENT;
+    const b200fft_sar_s* w = s->whole;
+    SarArgs a{};
+    a.in = raw_rows; a.out = nullptr; a.tw = w->tw_range;
+    a.tab = SarTables{w->H, w->mig, w->phs, w->stp};
+    a.tiles = s->g.pulses; a.ld = w->d.n_range; a.nr = (int)w->d.n_range; a.na = (int)w->d.n_azimuth; a.scale = 1.0f;
+    for (int g = 0; g < s->world; ++g) {
+        if (!strips[g]) return B200FFT_ERR_INVALID_ARG;
+        if (reinterpret_cast<uintptr_t>(strips[g]) % 16) return B200FFT_ERR_ALIGNMENT;
+        if (strips[g] == raw_rows) return B200FFT_ERR_INVALID_ARG;
+        a.sh.strip[g] = (unsigned long long)reinterpret_cast<uintptr_t>(strips[g]);
+    }
+    a.sh.world = s->world;
+    a.sh.strip_cols = (int)s->g.bins;
+    a.sh.halo_l = (int)s->g.halo_left;
+    a.sh.halo_r = (int)s->g.halo_right;
+    a.sh.sw = (int)s->g.strip_width;
+    a.sh.row0 = s->g.first_pulse;
+    return s->scatter->launch(a, reinterpret_cast<cudaStream_t>(stream)) == cudaSuccess ? B200FFT_OK : B200FFT_ERR_CUDA;
+}
+
+extern "C" int sar_rda_shard_azimuth(sar_rda_shard_t s, void* image_strip, void* stream) {
+    if (!s || !image_strip) return B200FFT_ERR_INVALID_ARG;
+    if (!s->strip->workspace) return B200FFT_ERR_WORKSPACE;
+    if (image_strip == s->strip->workspace) return B200FFT_ERR_INVALID_ARG;
+    int rc = sar_rda_run_step(nullptr, s->strip, image_strip, 1, stream);
+    if (rc != B200FFT_OK) return rc;
+    return sar_rda_run_step(nullptr, s->strip, image_strip, 2, stream);
+}
+
+extern "C" int sar_rda_shard_destroy(sar_rda_shard_t s) {
+    if (!s) return B200FFT_ERR_INVALID_ARG;
+    sar_rda_params_destroy(s->whole);
+    sar_rda_params_destroy(s->strip);
+    delete s;
     return B200FFT_OK;
 }

@@ -352,3 +352,72 @@ def test_shift_spread_at_the_edge_of_the_slab_guard(prf_hz, accepted):
     for dtype, tol in ((C64, 1e-5), (C32H, 5e-3)):
         for tile_columns in (2, 4):
             assert rel_l2(_gpu_chain(sc, raw, dtype, layout=1, tile_columns=tile_columns), img) <= tol
+
+
+def _gpu_sharded(scene, raw, dtype, world):
+    """The column-strip decomposition with all `world` ranks on one device: every rank's step 1 (range
+    compression scattered into every rank's strip buffer), then every rank's step 2 on its own strip."""
+    import torch
+    from paper_2609_32237_b200 import binding as B
+    desc = B.sar_desc_from_scene(scene, dtype)
+    shards = [B.sar_rda_shard_create(desc, r, world) for r in range(world)]
+    try:
+        geo = [B.sar_rda_shard_get_geometry(s) for s in shards]
+        for r, g in enumerate(geo):
+            h = B.sar_rda_shard_geometry_of(desc, r, world)
+            assert all(getattr(h, f) == getattr(g, f) for f, _ in B.SarShardGeometry._fields_)
+        # poisoned workspaces: whatever the kernels do not write shows up in the result
+        ws = [torch.full((g.workspace_bytes,), 0x7f, dtype=torch.uint8, device="cuda") for g in geo]
+        for s, w, g in zip(shards, ws, geo):
+            B.sar_rda_shard_set_workspace(s, w.data_ptr(), g.workspace_bytes)
+        rd = to_device_c64(raw)
+        ptrs = [w.data_ptr() for w in ws]
+        for r, (s, g) in enumerate(zip(shards, geo)):
+            rows = rd[g.first_pulse:g.first_pulse + g.pulses]
+            assert rows.is_contiguous()
+            B.sar_rda_shard_range_compress(s, rows.data_ptr(), ptrs, 0)
+        torch.cuda.synchronize()              # every rank's step 1 before any rank's step 2
+        image = np.zeros((scene.n_azimuth, scene.n_range), np.complex64)
+        for s, g in zip(shards, geo):
+            strip = torch.zeros(scene.n_azimuth, g.bins, 2, device="cuda")
+            B.sar_rda_shard_azimuth(s, strip.data_ptr(), 0)
+            torch.cuda.synchronize()
+            image[:, g.first_bin:g.first_bin + g.bins] = strip.cpu().numpy().view(np.complex64)[..., 0]
+        return image
+    finally:
+        for s in shards:
+            B.sar_rda_shard_destroy(s)
+
+
+@pytest.mark.parametrize("world", [1, 2, 4, 8])
+@pytest.mark.parametrize("dtype,tol", [(C64, 1e-5), (C32H, 5e-3)])
+def test_column_strip_decomposition_small_scene(small_scene, world, dtype, tol):
+    """Every rank count the decomposition accepts, all ranks emulated on one device: the assembled image against
+    the oracle and against the single-device chain; every target's peak cell."""
+    sc, raw, _, _, img = small_scene
+    got = _gpu_sharded(sc, raw, dtype, world)
+    assert rel_l2(got, img) <= tol
+    assert rel_l2(got, _gpu_chain(sc, raw, dtype)) <= (2e-6 if dtype == C64 else tol)
+    for cell in sc.targets:
+        assert quality.peak_cell(got, tuple(cell)) == tuple(cell)
+
+
+@pytest.mark.parametrize("world", [2, 8])
+def test_column_strip_decomposition_large_shifts(world, l_band_case):
+    """The L-band scene: the halo on the far side of every strip is about 200 bins wide."""
+    from paper_2609_32237_b200 import binding as B
+    sc, raw, img = l_band_case
+    g = B.sar_rda_shard_geometry_of(B.sar_desc_from_scene(sc, C64), 0, world)
+    assert g.halo_right >= 190 and g.halo_left == 8 and g.bins == sc.n_range // world
+    got = _gpu_sharded(sc, raw, C64, world)
+    assert rel_l2(got, img) <= 1e-5
+
+
+def test_column_strip_decomposition_refusals():
+    from paper_2609_32237_b200 import binding as B
+    sc = inputs.l_band_scene(n_azimuth=1024, n_range=1024, targets=[])
+    desc = B.sar_desc_from_scene(sc, C64)
+    for rank, world, status in ((0, 3, 1), (2, 2, 1), (-1, 2, 1), (0, 8, 2)):     # 8 strips of 128 bins: halos do not fit
+        with pytest.raises(B.B200FftError) as e:
+            B.sar_rda_shard_geometry_of(desc, rank, world)
+        assert e.value.status == status
