@@ -315,6 +315,47 @@ def time_cold(torch, fn, stream, scratch, steps, warmup, clean=False):
     return per
 
 
+def strips_one_rank(torch, B, sc, rd, dtype, world, stream, scratch, steps, whole_ms):
+    desc = B.sar_desc_from_scene(sc, dtype)
+    shards = [B.sar_rda_shard_create(desc, r, world) for r in range(world)]
+    geo = [B.sar_rda_shard_get_geometry(s) for s in shards]
+    ws = [torch.empty(int(g.workspace_bytes), dtype=torch.uint8, device="cuda") for g in geo]
+    for s_, w, g in zip(shards, ws, geo):
+        B.sar_rda_shard_set_workspace(s_, w.data_ptr(), int(g.workspace_bytes))
+    ptrs = [w.data_ptr() for w in ws]
+    strip = torch.empty(sc.n_azimuth, int(geo[0].bins), 2, device="cuda")
+    for r, (s_, g) in enumerate(zip(shards, geo)):          # every strip filled once, so that step 2 runs on real data
+        B.sar_rda_shard_range_compress(s_, rd[g.first_pulse:g.first_pulse + g.pulses].data_ptr(), ptrs, stream.cuda_stream)
+    torch.cuda.synchronize()
+    g0 = geo[0]
+    rows0 = rd[g0.first_pulse:g0.first_pulse + g0.pulses]
+    t1 = time_cold(torch, lambda: B.sar_rda_shard_range_compress(shards[0], rows0.data_ptr(), ptrs, stream.cuda_stream),
+                   stream, scratch, steps, 2)
+    def step2():
+        B.sar_rda_shard_azimuth(shards[0], strip.data_ptr(), stream.cuda_stream)
+        # the forward transform runs in place on the strip buffer: refill it outside the timed call
+    t2 = []
+    for i in range(steps + 2):
+        for r, (s_, g) in enumerate(zip(shards, geo)):
+            B.sar_rda_shard_range_compress(s_, rd[g.first_pulse:g.first_pulse + g.pulses].data_ptr(), ptrs, stream.cuda_stream)
+        flush_l2(torch, scratch)
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        step2()
+        b.record(stream)
+        torch.cuda.synchronize()
+        if i >= 2:
+            t2.append(a.elapsed_time(b))
+    for s_ in shards:
+        B.sar_rda_shard_destroy(s_)
+    rc_ms, az_ms = float(np.median(t1)), float(np.median(t2))
+    return {"range_compression_ms": rc_ms, "azimuth_steps_ms": az_ms, "sum_ms": rc_ms + az_ms,
+            "whole_image_on_one_device_ms": whole_ms, "ratio_to_whole": (rc_ms + az_ms) / whole_ms,
+            "halo_bins": [int(g0.halo_left), int(g0.halo_right)], "strip_bins": int(g0.bins),
+            "note": "one rank's two steps per image, all strip buffers on this device; the inter-device stores and "
+                    "the barrier between the steps are not in these numbers"}
+
+
 def bench_fft(torch, B, n, batch, dtype, seed, steps, warmup, layout="rows", direction=-1, cold_flush=None,
               options=None, also_clean=False):
     stream = torch.cuda.current_stream()
@@ -665,7 +706,15 @@ def run_others(torch, B, args, peak):
                             "d2h_bytes_per_image": raw.nbytes, "checksum": float(h_img.view(torch.float32)[:8].abs().sum())}
             B.sar_rda_params_destroy(p)
             out[base + suffix] = r
+            if not suffix:
+                default_ms = r["ms_median"]
             del ws
+        # Column-strip decomposition: what ONE rank of `world` does per image (its pulses' range compression,
+        # scattered into all strips, and the azimuth steps on its own strip), timed on this one device with
+        # every strip buffer local. The exchange between devices is not in these numbers.
+        for world in (2, 8):
+            out[f"{base}_column_strips_one_rank_of_{world}"] = strips_one_rank(torch, B, sc, rd, dtype, world, stream, scratch,
+                                                                                steps, default_ms)
     return out
 
 

@@ -421,3 +421,34 @@ def test_column_strip_decomposition_refusals():
         with pytest.raises(B.B200FftError) as e:
             B.sar_rda_shard_geometry_of(desc, rank, world)
         assert e.value.status == status
+
+
+def test_strip_rank_on_a_process_group_of_one(small_scene):
+    """The launcher for real devices (symmetric-memory strip buffers, barrier between the steps) with a
+    process group of one rank: both barrier styles, against the oracle."""
+    import os
+    import socket
+    import torch
+    import torch.distributed as dist
+    from paper_2609_32237_b200 import binding as B, multi
+    sc, raw, _, _, img = small_scene
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    os.environ["MASTER_ADDR"], os.environ["MASTER_PORT"] = "127.0.0.1", str(port)
+    torch.cuda.set_device(0)
+    dist.init_process_group("nccl", rank=0, world_size=1, device_id=torch.device("cuda", 0))
+    try:
+        rd = to_device_c64(raw)
+        for host_barrier in (True, False):
+            job = multi.SarStripRank(B.sar_desc_from_scene(sc, C64), host_barrier=host_barrier)
+            try:
+                assert job.geometry.pulses == sc.n_azimuth and job.geometry.bins == sc.n_range
+                out = job.form(rd)
+                torch.cuda.synchronize()
+                got = out.cpu().numpy().view(np.complex64)[..., 0]
+                assert rel_l2(got, img) <= 1e-5
+            finally:
+                job.close()
+    finally:
+        dist.destroy_process_group()
