@@ -123,7 +123,7 @@ int fft_plan_destroy(fft_plan_t plan);
  *   "stream"     (columns plans; "tma" is an alias) 1 selects the persistent streaming kernel (n = 2048
  *                complex64, n = 4096 both storage types): one CTA per multiprocessor loops over
  *                4-column tiles, and the tensor memory accelerator brings the next tile into shared
- *                memory (2-D tiled bulk copies of this GPU's own memory, no multicast) and takes the
+ *                memory (2-D tiled bulk copies of this GPU's own memory, each addressed to one CTA) and takes the
  *                finished one out while the current one is transformed; 0 forbids it; -1 restores the
  *                default rules.
  *   "staged"     (rows plans) n = 16384: 1 selects the persistent kernel whose next transform arrives

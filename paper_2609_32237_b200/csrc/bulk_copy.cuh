@@ -1,5 +1,5 @@
-// Thin wrappers over the tensor memory accelerator (2-D tiled cp.async.bulk.tensor and untiled
-// cp.async.bulk, no multicast) and mbarrier, as used by the TMA variant of the column-tile
+// Thin wrappers over the tensor memory accelerator (2-D tiled and untiled bulk copies, every one addressed to
+// the issuing CTA alone) and mbarrier, as used by the TMA variant of the column-tile
 // kernel and the staged persistent row kernel.
 #pragma once
 #include <cstdint>

@@ -18,7 +18,7 @@ namespace b200fft {
 // plain loads. After the last stage the results go back to shared memory as a dense image (the exchange
 // buffer is free by then) and leave as TMA stores, which the next tile's first stage overlaps; the stores
 // must have read shared memory before the next exchange overwrites it (wait_group.read). Tensor maps cover
-// this GPU's own memory; no multicast. Measured on 4096 x 4096 complex64: 74 us against 92 us for the plain
+// this GPU's own memory and every copy is addressed to the issuing CTA alone. Measured on 4096 x 4096 complex64: 74 us against 92 us for the plain
 // kernel. Variants that were built, tested and measured without gain, and dropped: two-column tiles at two CTAs
 // per multiprocessor, i.e. boxes with 16-byte rows (144 us); two warp groups of two columns each that take
 // turns on one 64 KiB exchange buffer, so that one group computes while the other exchanges, with the whole

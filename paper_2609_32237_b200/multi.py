@@ -33,7 +33,7 @@ class SarStripRank:
 
     The strip buffers live in symmetric memory so that every rank can address every other rank's
     buffer; the exchange itself is the epilogue of the range-compression kernel (plain stores to
-    the owners' buffers, nothing multicast), and the only synchronisation between the two steps is
+    the owners' buffers, every store addressed to one buffer), and the only synchronisation between the two steps is
     a barrier: on the device through the symmetric-memory signal pads (default), or on the host
     (`host_barrier=True`: stream synchronise, then the process group's barrier)."""
 
