@@ -113,8 +113,9 @@ int fft_plan_destroy(fft_plan_t plan);
  *                of length n2.
  *   "cluster"    c = 1, 2 or 4 (0 = the default rules; other values are B200FFT_ERR_INVALID_ARG): the
  *                single-pass variant in which c CTAs of one thread-block cluster share a tile through
- *                distributed shared memory. Defaults: rows of n = 16384 / 8192 with at most 32 / 16
- *                transforms, and rows of n = 32768, are split over clusters. Columns plans take, in
+ *                distributed shared memory. Defaults: rows of n = 16384 and n = 8192 with at most 32
+ *                transforms (4 CTAs each; n = 16384 up to 64 transforms: 2), and rows of n = 32768 (2),
+ *                are split over clusters. Columns plans take, in
  *                this order, the widest tile that is compiled and divides the batch: 16 columns for
  *                n <= 512 and 8 for n = 1024; the streaming kernel (see "stream") for n = 4096 when the
  *                matrix has more than one 4-column tile per multiprocessor; for other n >= 2048 a

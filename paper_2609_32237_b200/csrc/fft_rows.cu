@@ -174,12 +174,14 @@ int rows_stage_timeouts() {
 
 // Small batches leave most SMs idle with one CTA per transform (the paper's "when not to
 // use it"): there a transform is split over a cluster of CTAs through distributed shared
-// memory. Measured on B200: n = 16384, batch <= 32: 14.3 -> 10.2 us with 4 CTAs per transform;
-// n = 8192, batch <= 16: 12.3 -> 10.2 us with 2. Large batches are faster with one CTA.
+// memory. Measured on B200, device time per launch (replayed from a CUDA graph, data in L2):
+// n = 16384, batch <= 32: 8.2 us with one CTA per transform, 6.8 with 2, 5.1-5.6 with 4; batch 64: 8.5 / 7.2 / 7.6;
+// n = 8192, batch <= 32: 5.2 / 5.1 / 4.3-4.5; batch 64: 5.4 / 5.3 / 5.6. From a batch of 148 on one CTA wins.
 static int default_cluster(int n, int64_t batch) {
     if (n == 32768) return 2;
     if (n == 16384 && batch <= 32) return 4;
-    if (n == 8192 && batch <= 16) return 2;
+    if (n == 16384 && batch <= 64) return 2;
+    if (n == 8192 && batch <= 32) return 4;
     return 1;
 }
 

@@ -399,8 +399,9 @@ def test_execute_host_pipelined_and_simple_paths():
 
 def test_small_batches_pick_the_split_transform_variant():
     """Batches too small to fill the SMs default to a transform split over a cluster of
-    CTAs (N = 16384: batch <= 32; N = 8192: batch <= 16): parity at the switch-over sizes."""
-    for n, batch in ((16384, 32), (16384, 33), (8192, 16), (8192, 17), (16384, 2)):
+    CTAs (N = 16384: 4 CTAs up to batch 32, 2 up to 64; N = 8192: 4 CTAs up to batch 32): parity at the
+    switch-over sizes."""
+    for n, batch in ((16384, 32), (16384, 33), (16384, 64), (16384, 65), (8192, 32), (8192, 33), (16384, 2)):
         _check_rows(n, batch, seed=98, gaussian=True)
         _check_rows(n, batch, seed=99, direction=INV)
 
