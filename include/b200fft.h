@@ -254,7 +254,7 @@ int sar_rda_set_workspace(sar_rda_params_t params, void *device_ptr, size_t byte
  *                  intermediates and 4096 pulses the row pass writes a second fp16 image, one more rounding,
  *                  else the complex64 output on which the column pass then runs in place; the
  *                  default whenever the scene allows it: B200FFT_ERR_UNSUPPORTED if the migration grows
- *                  by more than 48 bins over 1024 range bins or n_range is not a multiple of 1024).
+ *                  by more than 112 bins over 2048 range bins).
  *   "layout"       0 (default) keeps the intermediate image row-major and transforms its columns
  *                  directly. 1 keeps it in slabs of 32-byte granules (4 complex64 or 8 complex-half range
  *                  bins; element (k, n) at ((n / G) * n_azimuth + k) * G + n % G), so that every column

@@ -301,12 +301,12 @@ def _noise_frame(n_azimuth, n_range, seed):
     return (g.standard_normal((n_azimuth, n_range)) + 1j * g.standard_normal((n_azimuth, n_range))).astype(np.complex64)
 
 
-@pytest.mark.parametrize("prf_hz,row_pass", [(986.0, True), (987.0, False), (1660.0, False)])
+@pytest.mark.parametrize("prf_hz,row_pass", [(1059.0, True), (1060.0, False), (1660.0, False)])
 def test_shift_growth_at_the_edge_of_the_row_pass_guard(prf_hz, row_pass):
-    """The row pass of step 2 stages 1024 + 64 range samples per CTA and is offered only while the
-    integer shift grows by at most 48 bins over 1024 range bins at the Doppler edge. With a 0.24 m
-    wavelength at 200 m/s that growth is 47.97 bins at PRF 986 Hz (accepted; shifts reach ~800 bins)
-    and 48.08 at 987 Hz (refused: step 2 falls back to the fused column kernel); 1660 Hz sits just
+    """The row pass of step 2 stages 2048 + 128 range samples per CTA and is offered only while the
+    integer shift grows by at most 112 bins over 2048 range bins at the Doppler edge. With a 0.24 m
+    wavelength at 200 m/s that growth is 111.9 bins at PRF 1059 Hz (accepted; shifts reach ~900 bins)
+    and 112.1 at 1060 Hz (refused: step 2 falls back to the fused column kernel); 1660 Hz sits just
     below the largest PRF the calls accept at all (shifts beyond the swath width). White noise as
     the raw frame makes every output pixel depend on the window it was read from."""
     from paper_2609_32237_b200 import binding as B
