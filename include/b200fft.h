@@ -313,8 +313,8 @@ int sar_rda_params_destroy(sar_rda_params_t params);
  * largest range migration of the frame plus the taps); halo bins outside the
  * frame are written as zeros by the rank that owns the pulse. The strip buffer
  * is the first strip_bytes of the rank's workspace (workspace_bytes in all).
- * world is 1, 2, 4 or 8; n_azimuth must be a multiple of world and n_range of
- * 8 * world; halo_left + halo_right must not exceed bins (else
+ * world is 1, 2, 4 or 8; n_azimuth must be a multiple of world, n_range / world a
+ * power of two (at least 8); halo_left + halo_right must not exceed bins (else
  * B200FFT_ERR_UNSUPPORTED). Results equal the single-device chain to rounding
  * (the per-bin coefficients are built in float64 for the strip's own origin).
  * ---------------------------------------------------------------------- */

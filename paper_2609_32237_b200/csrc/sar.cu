@@ -57,7 +57,7 @@ struct SarArgs {
     // store to: its own memory or a peer's). Bins outside the frame are written as zeros.
     struct {
         unsigned long long strip[8];
-        int world, strip_cols, halo_l, halo_r, sw;
+        int world, strip_cols, strip_shift, halo_l, halo_r, sw;   // strip_cols = 1 << strip_shift
         int64_t row0;    // first pulse of this launch within the whole frame
     } sh;
 };
@@ -113,7 +113,7 @@ __global__ void __launch_bounds__(C::THREADS, C::MINB) sar_range_compress_kernel
         const int64_t rowoff = (a.sh.row0 + tile) * (int64_t)a.sh.sw;      // this pulse's row in every strip
         auto strip = [&](int g) { return reinterpret_cast<void*>(a.sh.strip[g]); };
         e.template first_stage_dit_emit<true>(a.tw, 1.0f, [&](int p, int, float2 pa, float2 pb) {
-            const int g = p / sc, lc = p - g * sc;                       // sc, hl, hr are even: a pair stays together
+            const int g = p >> a.sh.strip_shift, lc = p & (sc - 1);     // sc, hl, hr are even: a pair stays together
             TOut::store2(strip(g), rowoff + hl + lc, pa, pb);
             if (lc < hr && g > 0) TOut::store2(strip(g - 1), rowoff + hl + sc + lc, pa, pb);
             if (lc >= sc - hl && g < last) TOut::store2(strip(g + 1), rowoff + lc - (sc - hl), pa, pb);
@@ -402,6 +402,7 @@ __global__ void __launch_bounds__(RcmcRows::TPB, TIn::ELEM_BYTES == 8 ? 6 : 5) s
 #pragma unroll
     for (int h = 0; h < COLS / (2 * TPB); ++h) {
         const int j = j0 + h * 2 * TPB + 2 * threadIdx.x;          // output columns j, j + 1
+        if (j >= a.out_cols) break;                                // a narrow strip ends inside the CTA's columns
         const int n = j + a.col0;                                  // range bins n, n + 1
         int ia, ib;
         float mua, mub;
@@ -449,7 +450,7 @@ __global__ void __launch_bounds__(RcmcRows::TPB, TIn::ELEM_BYTES == 8 ? 6 : 5) s
         const float2 fa = filter_phase(ph, n);
         const float2 fb = cmul(fa, step);
         const float2 ya = cmul(sa, fa), yb = cmul(sb, fb);
-        if (j < a.out_cols) TOut::store2(a.out, orow + j, ya, yb);
+        TOut::store2(a.out, orow + j, ya, yb);
     }
 }
 
@@ -1146,6 +1147,7 @@ extern "C" int sar_rda_shard_geometry_of(const sar_rda_desc* d, int32_t rank, in
         return B200FFT_ERR_INVALID_ARG;
     if (d->intermediate_dtype != B200FFT_C64 && d->intermediate_dtype != B200FFT_C32H) return B200FFT_ERR_INVALID_ARG;
     if (d->n_azimuth % world || d->n_range % (8 * world)) return B200FFT_ERR_UNSUPPORTED;
+    if ((d->n_range / world) & (d->n_range / world - 1)) return B200FFT_ERR_UNSUPPORTED;     // strips of 2^k bins
     const double wavelength = kLight / d->carrier_hz, dr = kLight / (2.0 * d->fs_hz);
     const double aa = wavelength * d->prf_hz / (4.0 * d->velocity_mps);
     if (aa >= 0.5) return B200FFT_ERR_INVALID_ARG;
@@ -1225,6 +1227,8 @@ extern "C" int sar_rda_shard_range_compress(sar_rda_shard_t s, const void* raw_r
     }
     a.sh.world = s->world;
     a.sh.strip_cols = (int)s->g.bins;
+    a.sh.strip_shift = 0;
+    while (((int64_t)1 << a.sh.strip_shift) < s->g.bins) ++a.sh.strip_shift;
     a.sh.halo_l = (int)s->g.halo_left;
     a.sh.halo_r = (int)s->g.halo_right;
     a.sh.sw = (int)s->g.strip_width;
