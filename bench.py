@@ -720,7 +720,7 @@ def run_others(torch, B, args, peak):
 
 def run_case(args):
     """One workload on its own (small JSON line): for profiling a single kernel.
-    --case rows:N:BATCH:c64|c32h[:inverse] | cols:N:BATCH:c64|c32h | sar:c64|c32h"""
+    --case rows:N:BATCH:c64|c32h[:inverse] | cols:N:BATCH:c64|c32h | sar:c64|c32h | sarstrips:c64|c32h"""
     import torch
     torch.cuda.set_device(0)
     from paper_2609_32237_b200 import binding as B
@@ -767,6 +767,45 @@ def run_case(args):
             cold[label] = round(float(np.median(ts[2:])) * 1e3, 1)
         out["cold_us"] = cold
         B.sar_rda_params_destroy(p)
+    elif kind == "sarstrips":
+        # The column-strip image formation on real devices, one process per GPU (torch.distributed.run sets
+        # RANK / LOCAL_RANK / WORLD_SIZE; without them: a process group of one). Per image: this rank's range
+        # compression with its stores into every rank's strip, a barrier, the azimuth steps on its strip, a barrier;
+        # device time per image, maximum over ranks.
+        import torch.distributed as dist
+        from paper_2609_32237_b200 import multi
+        dtype = dt[parts[1]]
+        rank, world = int(os.environ.get("RANK", "0")), int(os.environ.get("WORLD_SIZE", "1"))
+        local = int(os.environ.get("LOCAL_RANK", "0"))
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        os.environ.setdefault("MASTER_PORT", "29533")
+        torch.cuda.set_device(local)
+        dist.init_process_group("nccl", rank=rank, world_size=world, device_id=torch.device("cuda", local))
+        sc = inputs.x_band_scene()
+        job = multi.SarStripRank(B.sar_desc_from_scene(sc, dtype), host_barrier=any(o == "host_barrier=1" for o in args.option))
+        g = job.geometry
+        raw = inputs.simulate_raw(sc, seed=4)[g.first_pulse:g.first_pulse + g.pulses]
+        rows = torch.from_numpy(np.ascontiguousarray(raw)).cuda()
+        stream = torch.cuda.current_stream()
+        scratch = torch.empty(512 << 20, dtype=torch.uint8, device="cuda")
+        per = []
+        for i in range(args.warmup + args.steps):
+            flush_l2(torch, scratch)
+            dist.barrier()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            job.form(rows)
+            b.record(stream)
+            torch.cuda.synchronize()
+            if i >= args.warmup:
+                per.append(multi.max_over_ranks(a.elapsed_time(b), device="cuda"))
+        out = summarize(per, metrics.sar_bytes(4096, 4096, dtype), peak)
+        out["n_gpus"] = world
+        out["strip"] = {"bins": int(g.bins), "halo": [int(g.halo_left), int(g.halo_right)], "pulses": int(g.pulses)}
+        job.close()
+        dist.destroy_process_group()
+        if rank != 0:
+            return 0
     else:
         raise SystemExit(f"unknown case {args.case}")
     out["case"] = args.case
