@@ -120,3 +120,23 @@ def test_two_gloo_ranks_form_an_image_by_column_strips():
         assert p.exitcode == 0
     assert halo_right >= 190 and width == 8 + 512 + halo_right
     assert err <= 1e-11
+
+
+def test_strip_halos_cover_the_largest_migration_the_oracle_computes():
+    """halo_right of sar_rda_shard_geometry_of against the oracle's migration (in range bins) at the far
+    edge of the swath over every Doppler bin: the interpolator reads up to floor(migration) + 4 bins ahead."""
+    import math
+    import oracle
+    from paper_2609_32237_b200 import binding as B, inputs
+    for sc in (inputs.x_band_scene(n_azimuth=1024, n_range=2048, n_targets=0),
+               inputs.l_band_scene(n_azimuth=1024, n_range=2048, targets=[])):
+        p = oracle.sar_params(sc)
+        worst = max(oracle.sar_migration_bins(p, k, sc.n_range - 1) for k in range(sc.n_azimuth))
+        least = min(oracle.sar_migration_bins(p, k, 0) for k in range(sc.n_azimuth))
+        assert least >= 0.0                                   # the window never reaches further back than 3 bins
+        for world in (1, 2, 4):
+            g = B.sar_rda_shard_geometry_of(B.sar_desc_from_scene(sc, 0), world - 1, world)
+            assert g.halo_left >= 3
+            assert g.halo_right >= math.floor(worst) + 4
+            assert g.halo_right <= math.floor(worst) + 4 + 9  # rounded up to a multiple of 8, one bin of slack
+            assert g.halo_right % 8 == 0 and g.strip_width == g.halo_left + g.bins + g.halo_right
